@@ -1,0 +1,149 @@
+/*
+ * tsenor.h -- C ABI of the B200-native TSENOR hot path.
+ *
+ * TSENOR (arXiv 2505.23949) finds, for every aligned M x M block of a weight
+ * score matrix, a transposable N:M mask: a 0/1 block with exactly N ones in
+ * every row and every column that keeps as much score as possible (Eq. 1-2).
+ * It relaxes the block problem to a capacitated optimal-transport problem
+ * with an entropy term (Eq. 3-4), solves that with Dykstra's algorithm over
+ * the row-sum, column-sum and 0..1 box constraints (Algorithm 1, log domain
+ * as in Appendix A.2), and rounds the fractional plan with a greedy
+ * selection followed by a local search on the swap score of Eq. 6
+ * (Algorithm 2).
+ *
+ * Conventions shared by every entry point
+ *   - Every pointer is a DEVICE pointer owned by the caller unless the
+ *     comment says "host".  The library allocates nothing, never
+ *     synchronises, and enqueues all work on `stream`.
+ *   - Matrices are row-major fp32 with a leading dimension in elements
+ *     (`ld >= cols`).  |score| is taken inside; scores may have any sign.
+ *   - M is 4, 8, 16 or 32; rows and cols must be multiples of M.
+ *     Block (bi, bj) is the tile rows [bi*M, bi*M+M) x cols [bj*M, bj*M+M).
+ *   - A mask is `uint32_t[rows][tsenor_mask_words_per_row(cols)]`: bit
+ *     (c % 32) of word (c / 32) of row r is S[r][c]; bits past `cols` are 0.
+ *   - The return value is a host-side status decided before launch
+ *     (TSENOR_OK or a negative TSENOR_ERR_*).  Conditions found on the device
+ *     are OR-ed into the optional caller-owned `dev_status` word (the caller
+ *     zeroes it); kernels never trap and every device loop is bounded.
+ *   - tau is the paper's regularisation parameter: S(0) = exp(tau |W|).  The
+ *     library never guesses it.
+ */
+#ifndef TSENOR_H_
+#define TSENOR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Opaque CUDA stream handle (a cudaStream_t); NULL is the default stream. */
+typedef void *tsenor_stream_t;
+
+enum {
+    TSENOR_OK = 0,
+    TSENOR_ERR_NULL = -1,  /* a required pointer is NULL                      */
+    TSENOR_ERR_SHAPE = -2, /* negative size, ld < cols, rows/cols % M != 0    */
+    TSENOR_ERR_NM = -3,    /* M not in {4,8,16,32} or N outside its range     */
+    TSENOR_ERR_ARG = -4,   /* iters < 0, non-finite or negative tau, ...      */
+    TSENOR_ERR_CUDA = -5   /* launch failed: see tsenor_last_cuda_error()     */
+};
+
+/* Bits OR-ed into *dev_status by the kernels. */
+enum {
+    TSENOR_DEV_NONFINITE_SCORE = 1, /* a score or key was NaN/inf; masks of the
+                                       blocks holding one are unspecified      */
+    TSENOR_DEV_UNDERFILLED = 2,     /* some block ended with fewer than N per
+                                       line (only possible with ls_steps >= 0
+                                       or non-finite input)                    */
+    TSENOR_DEV_INTERNAL = 4         /* a bounded loop hit its limit            */
+};
+
+/*
+ * The whole method (Algorithm 1, then Algorithm 2) on every block, fused in
+ * one kernel: block loader, `iters` Dykstra iterations in fp32, greedy
+ * selection on the log-plan, local search, bit-packed mask.
+ *   scores        in   rows x cols fp32, leading dimension ld
+ *   N, M               0 <= N <= M (N = 0 / N = M give the all-zero / all-one mask)
+ *   tau                > 0 is the paper's setting; 0 allowed (uniform plan)
+ *   iters              T of Algorithm 1, >= 0 (0: greedy runs on tau|W| itself)
+ *   ls_steps           L of Algorithm 2.  < 0: repair until every line holds
+ *                      exactly N (best valid swap even if its score is <= 0;
+ *                      always terminates in M*N - |greedy| steps).  >= 0: the
+ *                      loop as printed (at most L steps, only swaps with a
+ *                      positive score).
+ *   mask_bits_out out  rows x words_per_row uint32, fully overwritten
+ *   dev_status    i/o  optional int32 status word (may be NULL)
+ */
+int tsenor_solve(const float *scores, int64_t rows, int64_t cols, int64_t ld,
+                 int N, int M, float tau, int iters, int ls_steps,
+                 uint32_t *mask_bits_out, int32_t *dev_status,
+                 tsenor_stream_t stream);
+
+/*
+ * Algorithm 1 alone (stage entry point for parity tests).  Requires
+ * 0 < N < M.  plan_out (rows x cols fp32, leading dimension ld_plan) receives
+ * S(T) = exp(x), or the log-plan x itself when plan_is_log != 0 (use the
+ * latter with iters == 0, where exp(tau|W|) may overflow fp32).
+ */
+int tsenor_dykstra(const float *scores, int64_t rows, int64_t cols, int64_t ld,
+                   int N, int M, float tau, int iters, float *plan_out,
+                   int64_t ld_plan, int plan_is_log, int32_t *dev_status,
+                   tsenor_stream_t stream);
+
+/*
+ * Algorithm 2 alone.  plan_key (rows x cols fp32, ld_plan) is any monotone
+ * image of the fractional plan; entries are taken in descending key order,
+ * equal keys in ascending flat index i*M+j inside the block (NaN keys order
+ * last, -0 equals +0).  The swap score of Eq. 6 is evaluated on |scores| in
+ * fp32 as (w[i][j'] + w[i'][j]) - w[i'][j'] with two roundings; the local
+ * search picks the lowest unsaturated row and column and breaks ties of the
+ * arg-max towards the smallest i'*M+j'.  Same mask layout, ls_steps and
+ * dev_status semantics as tsenor_solve.
+ */
+int tsenor_round(const float *plan_key, int64_t ld_plan, const float *scores,
+                 int64_t ld, int64_t rows, int64_t cols, int N, int M,
+                 int ls_steps, uint32_t *mask_bits_out, int32_t *dev_status,
+                 tsenor_stream_t stream);
+
+/*
+ * Objective of Eq. 1: *dev_sum_out (one double on the device, overwritten) =
+ * sum of |scores[r][c]| over the set bits of the mask, accumulated in fp64.
+ */
+int tsenor_objective(const float *scores, int64_t ld, const uint32_t *mask_bits,
+                     int64_t rows, int64_t cols, double *dev_sum_out,
+                     tsenor_stream_t stream);
+
+/*
+ * Feasibility of Eq. 2: *dev_bad_blocks_out (one int64 on the device,
+ * overwritten) = number of M x M blocks whose rows and columns do not all
+ * hold exactly N ones.
+ */
+int tsenor_check(const uint32_t *mask_bits, int64_t rows, int64_t cols, int N,
+                 int M, int64_t *dev_bad_blocks_out, tsenor_stream_t stream);
+
+/*
+ * *dev_max_out (one float on the device, overwritten) = max |scores[r][c]|
+ * (NaN entries are ignored).  Helper for the paper's parameter choice, which
+ * ties tau to the largest magnitude of the matrix (Appendix B.1).
+ */
+int tsenor_max_abs(const float *scores, int64_t rows, int64_t cols, int64_t ld,
+                   float *dev_max_out, tsenor_stream_t stream);
+
+/* ceil(cols / 32): uint32 words per mask row (host arithmetic only). */
+int64_t tsenor_mask_words_per_row(int64_t cols);
+
+/* Static description of a status returned by the functions above. */
+const char *tsenor_strerror(int status);
+
+/* cudaError_t value of the last failed launch on the calling thread (0 if none). */
+int tsenor_last_cuda_error(void);
+
+/* Kernels launched by this library (all threads) since it was loaded. */
+int64_t tsenor_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TSENOR_H_ */

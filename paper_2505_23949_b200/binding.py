@@ -1,0 +1,170 @@
+"""Thin Python binding of the C ABI in ``include/tsenor.h``: argument
+marshalling only.  Every step of the method runs in the CUDA kernels of
+``libtsenor.so``; there is no CPU fallback, and a missing library is an error.
+
+PyTorch is used for device memory and streams only.  Masks are returned as
+``torch.int32`` tensors holding the ``uint32`` words of the C ABI (bit
+``c % 32`` of word ``c // 32`` of row ``r`` is ``S[r, c]``).
+"""
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtsenor.so")
+
+OK, ERR_NULL, ERR_SHAPE, ERR_NM, ERR_ARG, ERR_CUDA = 0, -1, -2, -3, -4, -5
+DEV_NONFINITE_SCORE, DEV_UNDERFILLED, DEV_INTERNAL = 1, 2, 4
+
+EXPORTS = (
+    "tsenor_solve", "tsenor_dykstra", "tsenor_round", "tsenor_objective", "tsenor_check",
+    "tsenor_max_abs", "tsenor_mask_words_per_row", "tsenor_strerror", "tsenor_last_cuda_error",
+    "tsenor_launch_count",
+)
+
+_lib = None
+
+
+class TsenorError(RuntimeError):
+    def __init__(self, status, what):
+        self.status = status
+        msg = lib().tsenor_strerror(status).decode()
+        if status == ERR_CUDA:
+            msg += f" (cudaError {lib().tsenor_last_cuda_error()})"
+        super().__init__(f"{what}: {msg}")
+
+
+def lib():
+    """The loaded C-ABI library.  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2505_23949_b200.build` "
+                "(there is no fallback path)")
+        L = C.CDLL(LIB_PATH)
+        vp, i64, i32, f32 = C.c_void_p, C.c_int64, C.c_int, C.c_float
+        L.tsenor_solve.argtypes = [vp, i64, i64, i64, i32, i32, f32, i32, i32, vp, vp, vp]
+        L.tsenor_dykstra.argtypes = [vp, i64, i64, i64, i32, i32, f32, i32, vp, i64, i32, vp, vp]
+        L.tsenor_round.argtypes = [vp, i64, vp, i64, i64, i64, i32, i32, i32, vp, vp, vp]
+        L.tsenor_objective.argtypes = [vp, i64, vp, i64, i64, vp, vp]
+        L.tsenor_check.argtypes = [vp, i64, i64, i32, i32, vp, vp]
+        L.tsenor_max_abs.argtypes = [vp, i64, i64, i64, vp, vp]
+        for name in ("tsenor_solve", "tsenor_dykstra", "tsenor_round", "tsenor_objective",
+                     "tsenor_check", "tsenor_max_abs", "tsenor_last_cuda_error"):
+            getattr(L, name).restype = i32
+        L.tsenor_mask_words_per_row.argtypes = [i64]
+        L.tsenor_mask_words_per_row.restype = i64
+        L.tsenor_strerror.argtypes = [i32]
+        L.tsenor_strerror.restype = C.c_char_p
+        L.tsenor_launch_count.argtypes = []
+        L.tsenor_launch_count.restype = i64
+        _lib = L
+    return _lib
+
+
+def _stream(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def _mat(t, name):
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.float32 and t.dim() == 2):
+        raise TypeError(f"{name} must be a 2-D float32 CUDA tensor")
+    if t.stride(1) != 1:
+        raise ValueError(f"{name} must be row-major (unit column stride)")
+    ld = t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1])
+    return t.data_ptr(), t.shape[0], t.shape[1], ld
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def mask_words_per_row(cols):
+    return int(lib().tsenor_mask_words_per_row(int(cols)))
+
+
+def new_mask(rows, cols, device):
+    return torch.empty((rows, mask_words_per_row(cols)), dtype=torch.int32, device=device)
+
+
+def new_status(device):
+    return torch.zeros(1, dtype=torch.int32, device=device)
+
+
+def launch_count():
+    return int(lib().tsenor_launch_count())
+
+
+def solve(scores, N, M, tau, iters=300, ls_steps=-1, mask_out=None, status=None, stream=None):
+    """tsenor_solve: Algorithm 1 + Algorithm 2 on every M x M block.  Asynchronous."""
+    p, rows, cols, ld = _mat(scores, "scores")
+    if mask_out is None:
+        mask_out = new_mask(rows, cols, scores.device)
+    rc = lib().tsenor_solve(p, rows, cols, ld, int(N), int(M), float(tau), int(iters), int(ls_steps),
+                            _ptr(mask_out), _ptr(status), _stream(stream))
+    if rc:
+        raise TsenorError(rc, "tsenor_solve")
+    return mask_out
+
+
+def dykstra(scores, N, M, tau, iters=300, plan_is_log=False, plan_out=None, status=None, stream=None):
+    """tsenor_dykstra: Algorithm 1 only; returns the fp32 plan (or log-plan)."""
+    p, rows, cols, ld = _mat(scores, "scores")
+    if plan_out is None:
+        plan_out = torch.empty((rows, cols), dtype=torch.float32, device=scores.device)
+    pp, _, _, ldp = _mat(plan_out, "plan_out")
+    rc = lib().tsenor_dykstra(p, rows, cols, ld, int(N), int(M), float(tau), int(iters), pp, ldp,
+                              int(bool(plan_is_log)), _ptr(status), _stream(stream))
+    if rc:
+        raise TsenorError(rc, "tsenor_dykstra")
+    return plan_out
+
+
+def round_plan(plan_key, scores, N, M, ls_steps=-1, mask_out=None, status=None, stream=None):
+    """tsenor_round: Algorithm 2 only, from fp32 keys and fp32 scores."""
+    pk, rows, cols, ldk = _mat(plan_key, "plan_key")
+    ps, r2, c2, ld = _mat(scores, "scores")
+    if (rows, cols) != (r2, c2):
+        raise ValueError("plan_key and scores differ in shape")
+    if mask_out is None:
+        mask_out = new_mask(rows, cols, scores.device)
+    rc = lib().tsenor_round(pk, ldk, ps, ld, rows, cols, int(N), int(M), int(ls_steps),
+                            _ptr(mask_out), _ptr(status), _stream(stream))
+    if rc:
+        raise TsenorError(rc, "tsenor_round")
+    return mask_out
+
+
+def objective(scores, mask, out=None, stream=None):
+    """tsenor_objective: 1-element float64 device tensor with the retained score."""
+    p, rows, cols, ld = _mat(scores, "scores")
+    if out is None:
+        out = torch.empty(1, dtype=torch.float64, device=scores.device)
+    rc = lib().tsenor_objective(p, ld, _ptr(mask), rows, cols, _ptr(out), _stream(stream))
+    if rc:
+        raise TsenorError(rc, "tsenor_objective")
+    return out
+
+
+def check(mask, rows, cols, N, M, out=None, stream=None):
+    """tsenor_check: 1-element int64 device tensor with the number of infeasible blocks."""
+    if out is None:
+        out = torch.empty(1, dtype=torch.int64, device=mask.device)
+    rc = lib().tsenor_check(_ptr(mask), int(rows), int(cols), int(N), int(M), _ptr(out), _stream(stream))
+    if rc:
+        raise TsenorError(rc, "tsenor_check")
+    return out
+
+
+def max_abs(scores, out=None, stream=None):
+    """tsenor_max_abs: 1-element float32 device tensor with max |score|."""
+    p, rows, cols, ld = _mat(scores, "scores")
+    if out is None:
+        out = torch.empty(1, dtype=torch.float32, device=scores.device)
+    rc = lib().tsenor_max_abs(p, rows, cols, ld, _ptr(out), _stream(stream))
+    if rc:
+        raise TsenorError(rc, "tsenor_max_abs")
+    return out

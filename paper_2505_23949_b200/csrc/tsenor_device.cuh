@@ -1,0 +1,597 @@
+// Device code of the TSENOR hot path for sm_100a: block loader, log-domain
+// Dykstra iterations (Algorithm 1), greedy selection and local search
+// (Algorithm 2, Eq. 6), bit-packed mask writer.
+//
+// Layout in one sentence: a CTA owns a panel of M rows x PANEL columns of the
+// score matrix (PANEL = WARPS * BPW * M), stages it in shared memory with
+// coalesced loads, every warp runs Dykstra for its BPW blocks entirely in
+// registers, hands the log-plan to the rounding stage through shared memory,
+// and the CTA writes whole 32-bit mask words back.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace tsenor {
+
+constexpr unsigned FULL = 0xffffffffu;
+constexpr int WARPS = 4;  // warps per CTA
+
+enum : int { DEV_NONFINITE = 1, DEV_UNDERFILLED = 2, DEV_INTERNAL = 4 };
+
+// ---------------------------------------------------------------------------
+// Dykstra register layout.  A block is spread over LPB = PR*PC lanes arranged
+// as PR x PC; each lane keeps an MR x MC sub-tile (4 x 8 floats, 4 x 4 for
+// M = 4).  Row sums are reduced over the PC lanes that share rows, column
+// sums over the PR lanes that share columns.
+// ---------------------------------------------------------------------------
+template <int M> struct Tile;
+template <> struct Tile<32> { static constexpr int PR = 8, PC = 4, MR = 4, MC = 8; };
+template <> struct Tile<16> { static constexpr int PR = 4, PC = 2, MR = 4, MC = 8; };
+template <> struct Tile<8>  { static constexpr int PR = 2, PC = 1, MR = 4, MC = 8; };
+template <> struct Tile<4>  { static constexpr int PR = 1, PC = 1, MR = 4, MC = 4; };
+
+template <int M> struct Geom {
+    using T = Tile<M>;
+    static constexpr int LPB = T::PR * T::PC;        // lanes per block (Dykstra)
+    static constexpr int BPW = 32 / LPB;             // blocks per warp
+    static constexpr int PANEL = WARPS * BPW * M;    // panel width in columns
+    static constexpr int WS = PANEL + 1;             // shared row stride (floats)
+    static constexpr int GPW = 32 / M;               // rounding groups per warp
+    static constexpr int PASSES = BPW / GPW;         // rounding passes per warp
+    static constexpr int TS = M + 4;                 // byte-table row stride
+    static constexpr int WORDS = PANEL / 32;         // mask words per panel row
+};
+
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float lg2_approx(float x) {
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float rcp_approx(float x) {
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Register r of a lane holds line (r ^ perm) of its sub-tile, where perm is
+// built from the lane's coordinate along the reduction direction.  With that
+// permutation the recursive-halving exchange below needs no selects: every
+// lane always sends its upper half and keeps its lower half.
+template <int K, int P> __device__ __forceinline__ int xor_perm(int l) {
+    int g = 0;
+#pragma unroll
+    for (int s = 0; (1 << s) < P; ++s) g |= ((l >> s) & 1) * (K >> (s + 1));
+    return g;
+}
+
+struct OpAdd { __device__ __forceinline__ float operator()(float a, float b) const { return a + b; } };
+struct OpMax { __device__ __forceinline__ float operator()(float a, float b) const { return fmaxf(a, b); } };
+
+// After the call v[0 .. K/P) hold the reduction over the P lanes (lane stride
+// `base`) of the lines those registers stand for.
+template <int K, int P, class Op>
+__device__ __forceinline__ void reduce_scatter(float (&v)[K], int base, Op op) {
+#pragma unroll
+    for (int s = 0; (1 << s) < P; ++s) {
+        const int h = K >> (s + 1);
+#pragma unroll
+        for (int k = 0; k < h; ++k)
+            v[k] = op(v[k], __shfl_xor_sync(FULL, v[k + h], base << s));
+    }
+}
+// Inverse exchange: v[0 .. K/P) valid on entry, all K valid on return.
+template <int K, int P>
+__device__ __forceinline__ void all_gather(float (&v)[K], int base) {
+    constexpr int S = (P == 1) ? 0 : (P == 2) ? 1 : (P == 4) ? 2 : 3;
+#pragma unroll
+    for (int s = S - 1; s >= 0; --s) {
+        const int h = K >> (s + 1);
+#pragma unroll
+        for (int k = 0; k < h; ++k)
+            v[k + h] = __shfl_xor_sync(FULL, v[k], base << s);
+    }
+}
+
+// Kahan-compensated running sum for the few potentials a lane owns.
+struct Comp {
+    float hi, lo;
+    __device__ __forceinline__ void add(float a) {
+        float y = a - lo;
+        float t = hi + y;
+        lo = (t - hi) - y;
+        hi = t;
+    }
+};
+
+// ---------------------------------------------------------------------------
+// Algorithm 1 in potential form.
+//
+// In the log domain the three projections only ever add a row term and a
+// column term to x + q, and after the clip x = min(t, 0), q = max(t, 0) for
+// t = x + q.  So the whole state is t_ij = t0_ij + F_i + G_j with
+// t0 = tau |w| (base-2 units here), and one iteration is
+//     e_ij   = min(2^t_ij, 1)                      (S of the previous clip)
+//     F_i   += log2 N - log2 sum_j e_ij            (projection on C1)
+//     G_j   += log2 N - log2 sum_i e_ij N / r_i    (projection on C2)
+// with the clip (C3) and the dual update implicit in the next e.  One exp per
+// element and iteration.  Iteration 0 has no clip yet and its column pass is
+// done with the maximum subtracted, because 2^t0 of a whole column can
+// underflow against a large entry elsewhere in its rows; from iteration 1 on
+// every row and column sum is bounded below by N/M, so no sum can vanish.
+// On entry t holds t0 with its row maximum subtracted (exact no-op for the
+// method: the first row projection removes any row constant); on return t
+// holds the final t = x + q.
+// ---------------------------------------------------------------------------
+template <int M>
+__device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>::MC], int lane_in_blk,
+                                                float Nf, float log2N, int iters) {
+    using T = Tile<M>;
+    constexpr int MR = T::MR, MC = T::MC, PR = T::PR, PC = T::PC;
+    constexpr int RO = MR / PC, CO = MC / PR;  // lines whose sums this lane finishes
+    (void)lane_in_blk;
+    float F[MR], G[MC];
+    Comp Fo[RO], Go[CO];
+    if (iters <= 0) return;
+    {   // iteration 0
+        float rp[MR];
+#pragma unroll
+        for (int a = 0; a < MR; ++a) {
+            float s = 0.f;
+#pragma unroll
+            for (int b = 0; b < MC; ++b) s += ex2_approx(t[a][b]);
+            rp[a] = s;
+        }
+        reduce_scatter<MR, PC>(rp, 1, OpAdd());
+#pragma unroll
+        for (int k = 0; k < RO; ++k) {
+            Fo[k].hi = log2N - lg2_approx(rp[k]);
+            Fo[k].lo = 0.f;
+            F[k] = Fo[k].hi;
+        }
+        all_gather<MR, PC>(F, 1);
+        float cm[MC];
+#pragma unroll
+        for (int b = 0; b < MC; ++b) {
+            float m = t[0][b] + F[0];
+#pragma unroll
+            for (int a = 1; a < MR; ++a) m = fmaxf(m, t[a][b] + F[a]);
+            cm[b] = m;
+        }
+        reduce_scatter<MC, PR>(cm, PC, OpMax());
+        all_gather<MC, PR>(cm, PC);
+        float cp[MC];
+#pragma unroll
+        for (int b = 0; b < MC; ++b) {
+            float s = 0.f;
+#pragma unroll
+            for (int a = 0; a < MR; ++a) s += ex2_approx((t[a][b] + F[a]) - cm[b]);
+            cp[b] = s;
+        }
+        reduce_scatter<MC, PR>(cp, PC, OpAdd());
+#pragma unroll
+        for (int k = 0; k < CO; ++k) {
+            Go[k].hi = (log2N - cm[k]) - lg2_approx(cp[k]);
+            Go[k].lo = 0.f;
+            G[k] = Go[k].hi;
+        }
+        all_gather<MC, PR>(G, PC);
+    }
+    for (int it = 1; it < iters; ++it) {
+        float e[MR][MC], rp[MR], rho[MR], cp[MC];
+#pragma unroll
+        for (int a = 0; a < MR; ++a) {
+            float s = 0.f;
+#pragma unroll
+            for (int b = 0; b < MC; ++b) {
+                e[a][b] = fminf(ex2_approx((t[a][b] + F[a]) + G[b]), 1.0f);
+                s += e[a][b];
+            }
+            rp[a] = s;
+        }
+        reduce_scatter<MR, PC>(rp, 1, OpAdd());
+#pragma unroll
+        for (int k = 0; k < RO; ++k) {
+            rho[k] = Nf * rcp_approx(rp[k]);
+            Fo[k].add(log2N - lg2_approx(rp[k]));
+            F[k] = Fo[k].hi;
+        }
+        all_gather<MR, PC>(rho, 1);
+        all_gather<MR, PC>(F, 1);
+#pragma unroll
+        for (int b = 0; b < MC; ++b) {
+            float s = e[0][b] * rho[0];
+#pragma unroll
+            for (int a = 1; a < MR; ++a) s = fmaf(e[a][b], rho[a], s);
+            cp[b] = s;
+        }
+        reduce_scatter<MC, PR>(cp, PC, OpAdd());
+#pragma unroll
+        for (int k = 0; k < CO; ++k) {
+            Go[k].add(log2N - lg2_approx(cp[k]));
+            G[k] = Go[k].hi;
+        }
+        all_gather<MC, PR>(G, PC);
+    }
+#pragma unroll
+    for (int a = 0; a < MR; ++a)
+#pragma unroll
+        for (int b = 0; b < MC; ++b) t[a][b] = (t[a][b] + F[a]) + G[b];
+}
+
+// ---------------------------------------------------------------------------
+// Panel loader: |score| of an M x PANEL panel into shared memory, coalesced,
+// 16-byte vector loads when the addresses allow it.  Returns non-zero if a
+// non-finite value was seen by this thread.
+// ---------------------------------------------------------------------------
+template <int M>
+__device__ __forceinline__ int load_panel(const float* __restrict__ src, int64_t ld, int64_t r0, int64_t c0,
+                                          int64_t cols, bool vec_ok, bool take_abs, float* __restrict__ dst) {
+    using G = Geom<M>;
+    constexpr int V = G::PANEL / 4;
+    int bad = 0;
+    for (int idx = threadIdx.x; idx < M * V; idx += WARPS * 32) {
+        const int r = idx / V, c = (idx % V) * 4;
+        const int64_t gc = c0 + c;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (gc < cols) {  // cols is a multiple of 4, so a quad is all in or all out
+            const float* p = src + (r0 + r) * ld + gc;
+            if (vec_ok) {
+                v = __ldg(reinterpret_cast<const float4*>(p));
+            } else {
+                v.x = __ldg(p); v.y = __ldg(p + 1); v.z = __ldg(p + 2); v.w = __ldg(p + 3);
+            }
+        }
+        if (take_abs) { v.x = fabsf(v.x); v.y = fabsf(v.y); v.z = fabsf(v.z); v.w = fabsf(v.w); }
+        bad |= !(fabsf(v.x) <= 3.4028234e38f) | !(fabsf(v.y) <= 3.4028234e38f) |
+               !(fabsf(v.z) <= 3.4028234e38f) | !(fabsf(v.w) <= 3.4028234e38f);
+        float* d = dst + r * G::WS + c;
+        d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
+    }
+    return bad;
+}
+
+// ---------------------------------------------------------------------------
+// Rounding stage (Algorithm 2).  A group of M lanes owns one block; lane i of
+// the group plays row i and column i at once.
+// ---------------------------------------------------------------------------
+template <int M> struct RoundTables {
+    static constexpr int TS = Geom<M>::TS;
+    unsigned char rperm[M * TS];  // [i][p] -> column of the p-th best entry of row i
+    unsigned char cperm[M * TS];  // [j][s] -> row of the s-th best entry of column j
+    unsigned char rrank[M * TS];  // [i][j] -> rank of (i,j) inside row i
+    unsigned char crank[M * TS];  // [j][i] -> rank of (i,j) inside column j
+    unsigned int rs[M];           // row-side picks of the round, bits over columns
+    unsigned int cs[M];           // column-side picks of the round, bits over rows
+    unsigned int sel[M];          // current mask, one word per row
+};
+
+// Strict order "key descending, index ascending" as one ascending u64.
+__device__ __forceinline__ unsigned long long sort_word(float key, int idx) {
+    if (!(key == key)) key = __int_as_float(0xff800000);  // NaN orders as -inf
+    key += 0.0f;                                          // -0 -> +0
+    unsigned u = __float_as_uint(key);
+    u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);       // ascending uint == ascending float
+    return ((unsigned long long)(~u) << 32) | (unsigned)idx;
+}
+
+template <int M> __device__ __forceinline__ void sort_regs(unsigned long long (&v)[M]) {
+#pragma unroll
+    for (int k = 2; k <= M; k <<= 1)
+#pragma unroll
+        for (int j = k >> 1; j > 0; j >>= 1)
+#pragma unroll
+            for (int i = 0; i < M; ++i) {
+                const int l = i ^ j;
+                if (l > i) {
+                    const bool up = ((i & k) == 0);
+                    const unsigned long long a = v[i], b = v[l];
+                    const bool sw = up ? (a > b) : (a < b);
+                    v[i] = sw ? b : a;
+                    v[l] = sw ? a : b;
+                }
+            }
+}
+
+// Sorts one line (stride `st` floats in shared memory) and writes the
+// permutation and rank tables for it.
+template <int M>
+__device__ __forceinline__ void sort_line(const float* line, int st, unsigned char* perm, unsigned char* rank) {
+    unsigned long long v[M];
+#pragma unroll
+    for (int k = 0; k < M; ++k) v[k] = sort_word(line[k * st], k);
+    sort_regs<M>(v);
+#pragma unroll
+    for (int p = 0; p < M; ++p) {
+        const int k = (int)(v[p] & 63u);
+        perm[p] = (unsigned char)k;
+        rank[k] = (unsigned char)p;
+    }
+}
+
+// Greedy selection + local search for the block of this lane's group.
+//   ks, ws: shared-memory pointers to element (0,0) of the block's keys and
+//   |scores| (row stride WS); tb: the group's tables; active: group has a block.
+// Returns this lane's row of the mask (M bits).  flags accumulates DEV_* bits.
+template <int M>
+__device__ __forceinline__ unsigned round_block(const float* ks, const float* ws, RoundTables<M>& tb, int lane,
+                                                bool active, int N, int ls_steps, int& flags) {
+    using G = Geom<M>;
+    constexpr int WS = G::WS, TS = G::TS;
+    constexpr unsigned GM = (M == 32) ? 0xffffffffu : ((1u << (M & 31)) - 1u);
+    const int i = lane % M;            // my row, and my column
+    const int gsh = (lane / M) * M;    // first lane of my group
+
+    // ---- sorted orders of my row and of my column (Algorithm 2 line 2)
+    sort_line<M>(ks + i * WS, 1, tb.rperm + i * TS, tb.rrank + i * TS);
+    sort_line<M>(ks + i, WS, tb.cperm + i * TS, tb.crank + i * TS);
+    __syncwarp();
+
+    // ---- greedy selection (lines 3-6) in synchronous rounds.  An available
+    // entry (not taken, row and column not full) that ranks below the
+    // remaining capacity among the available entries of both its row and its
+    // column is taken by the sequential scan whatever happens elsewhere, so
+    // all such entries are taken at once; the first available entry in the
+    // global order always qualifies, hence every round makes progress and the
+    // fixed point is the sequential result.
+    unsigned A = active ? GM : 0u, B = A;   // available entries, rank space
+    int capR = active ? N : 0, capC = capR;
+    bool rowdone = !active, coldone = !active;
+    unsigned sel = 0u;
+    for (int round = 0; round < M * M; ++round) {
+        if (!__any_sync(FULL, A != 0u)) break;
+        if (round == M * M - 1) flags |= DEV_INTERNAL;
+        // picks: the first capR (capC) available entries in rank order
+        unsigned ar = A, bc = B, pickR = 0u, pickC = 0u, RS = 0u, CS = 0u;
+        int nr = capR, nc = capC;
+        while (__any_sync(FULL, (nr > 0 && ar) || (nc > 0 && bc))) {
+            if (nr > 0 && ar) {
+                const int p = __ffs(ar) - 1;
+                ar &= ar - 1; --nr;
+                pickR |= 1u << p;
+                RS |= 1u << tb.rperm[i * TS + p];
+            }
+            if (nc > 0 && bc) {
+                const int s = __ffs(bc) - 1;
+                bc &= bc - 1; --nc;
+                pickC |= 1u << s;
+                CS |= 1u << tb.cperm[i * TS + s];
+            }
+        }
+        tb.rs[i] = RS;
+        tb.cs[i] = CS;
+        __syncwarp();
+        // an entry picked from both sides is taken
+        while (__any_sync(FULL, pickR | pickC)) {
+            if (pickR) {
+                const int p = __ffs(pickR) - 1;
+                pickR &= pickR - 1;
+                const int j = tb.rperm[i * TS + p];
+                if ((tb.cs[j] >> i) & 1u) { sel |= 1u << j; A &= ~(1u << p); --capR; }
+            }
+            if (pickC) {
+                const int s = __ffs(pickC) - 1;
+                pickC &= pickC - 1;
+                const int r = tb.cperm[i * TS + s];
+                if ((tb.rs[r] >> i) & 1u) { B &= ~(1u << s); --capC; }
+            }
+        }
+        __syncwarp();
+        // lines that just filled up drop out, and so do their entries
+        const bool rfull = (capR == 0) && !rowdone, cfull = (capC == 0) && !coldone;
+        unsigned nfr = (__ballot_sync(FULL, rfull) >> gsh) & GM;
+        unsigned nfc = (__ballot_sync(FULL, cfull) >> gsh) & GM;
+        if (rfull) { A = 0u; rowdone = true; }
+        if (cfull) { B = 0u; coldone = true; }
+        while (__any_sync(FULL, nfr | nfc)) {
+            if (nfr) {
+                const int r = __ffs(nfr) - 1;
+                nfr &= nfr - 1;
+                B &= ~(1u << tb.crank[i * TS + r]);
+            }
+            if (nfc) {
+                const int c = __ffs(nfc) - 1;
+                nfc &= nfc - 1;
+                A &= ~(1u << tb.rrank[i * TS + c]);
+            }
+        }
+    }
+
+    // ---- local search (lines 7-13, Eq. 6).  Lane j' scans i' = 0..M-1.
+    tb.sel[i] = sel;
+    __syncwarp();
+    bool stopped = !active;
+    int steps = 0;
+    for (int it = 0; it <= M * N; ++it) {
+        const unsigned rdef = (__ballot_sync(FULL, capR > 0) >> gsh) & GM;
+        const unsigned cdef = (__ballot_sync(FULL, capC > 0) >> gsh) & GM;
+        const bool work = !stopped && rdef != 0u && cdef != 0u && (ls_steps < 0 || steps < ls_steps);
+        if (!__any_sync(FULL, work)) break;
+        if (it == M * N) { flags |= DEV_INTERNAL; break; }
+        const int di = work ? __ffs(rdef) - 1 : 0;   // lowest unsaturated row
+        const int dj = work ? __ffs(cdef) - 1 : 0;   // lowest unsaturated column
+        const int jp = i;                            // my candidate column j'
+        float best = __int_as_float(0xff800000);
+        int bi = 0x7fffffff;
+        if (work && !((tb.sel[di] >> jp) & 1u)) {
+            const float w_ijp = ws[di * WS + jp];
+#pragma unroll 4
+            for (int ip = 0; ip < M; ++ip) {
+                const unsigned s = tb.sel[ip];
+                const bool valid = ((s >> jp) & 1u) && !((s >> dj) & 1u);
+                const float sc = __fsub_rn(__fadd_rn(w_ijp, ws[ip * WS + dj]), ws[ip * WS + jp]);
+                if (valid && sc > best) { best = sc; bi = ip; }
+            }
+        }
+        int bflat = (bi == 0x7fffffff) ? 0x7fffffff : bi * M + jp;
+#pragma unroll
+        for (int off = M / 2; off > 0; off >>= 1) {
+            const float ob = __shfl_xor_sync(FULL, best, off, M);
+            const int of = __shfl_xor_sync(FULL, bflat, off, M);
+            if (ob > best || (ob == best && of < bflat)) { best = ob; bflat = of; }
+        }
+        if (work) {
+            if (bflat == 0x7fffffff) {            // no valid triple: only with non-finite scores
+                stopped = true;
+            } else if (ls_steps >= 0 && !(best > 0.0f)) {
+                stopped = true;                   // paper-strict loop: improving swaps only
+            } else {
+                const int ip = bflat / M, jq = bflat % M;
+                if (i == ip) sel = (sel & ~(1u << jq)) | (1u << dj);
+                if (i == di) { sel |= 1u << jq; --capR; }
+                if (i == dj) --capC;
+                ++steps;
+            }
+        }
+        __syncwarp();
+        tb.sel[i] = sel;
+        __syncwarp();
+    }
+    if (active && (capR != 0 || capC != 0)) flags |= DEV_UNDERFILLED;
+    return sel;
+}
+
+// ---------------------------------------------------------------------------
+// Fused kernel.  MODE 0: whole method; 1: Algorithm 1 only (plan to global);
+// 2: Algorithm 2 only (keys from global).
+// ---------------------------------------------------------------------------
+struct Params {
+    const float* scores; int64_t ld;
+    const float* keys;   int64_t ld_keys;
+    float* plan;         int64_t ld_plan; int plan_is_log;
+    uint32_t* bits;      int64_t wpr;
+    int64_t rows, cols;
+    int npc;                       // panels per block row
+    int N; float Nf, log2N;
+    float c_hi, c_lo;              // tau * log2(e), split in two floats
+    int iters, ls_steps;
+    int32_t* status;
+    int vec_scores, vec_keys;
+};
+
+template <int M> struct SmemLayout {
+    using G = Geom<M>;
+    float w[M * G::WS];
+    float k[M * G::WS];
+    RoundTables<M> tb[WARPS * G::GPW];
+    unsigned int bits[M * G::WORDS];
+};
+
+template <int M, int MODE>
+__global__ void __launch_bounds__(WARPS * 32) tsenor_kernel(const Params P) {
+    using G = Geom<M>;
+    using T = Tile<M>;
+    constexpr int MR = T::MR, MC = T::MC, PR = T::PR, PC = T::PC;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    SmemLayout<M>& sm = *reinterpret_cast<SmemLayout<M>*>(smem_raw);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t panel = blockIdx.x;
+    const int64_t r0 = (panel / P.npc) * M;
+    const int64_t c0 = (panel % P.npc) * (int64_t)G::PANEL;
+    const int valid_cols = (int)((P.cols - c0 < G::PANEL) ? (P.cols - c0) : G::PANEL);
+    int flags = 0;
+
+    // ---- block loader
+    if (load_panel<M>(P.scores, P.ld, r0, c0, P.cols, P.vec_scores != 0, true, sm.w)) flags |= DEV_NONFINITE;
+    if (MODE == 2)
+        if (load_panel<M>(P.keys, P.ld_keys, r0, c0, P.cols, P.vec_keys != 0, false, sm.k)) flags |= DEV_NONFINITE;
+    if (MODE != 1)
+        for (int idx = threadIdx.x; idx < M * G::WORDS; idx += WARPS * 32) sm.bits[idx] = 0u;
+    __syncthreads();
+
+    // ---- Algorithm 1
+    if (MODE != 2) {
+        const int g = lane % G::LPB;                          // lane inside its block
+        const int blk = warp * G::BPW + lane / G::LPB;        // block inside the panel
+        const int lr = g / PC, lc = g % PC;
+        const int gr = xor_perm<MR, PC>(lc), gc = xor_perm<MC, PR>(lr);
+        const bool active = blk * M < valid_cols;
+        float t[MR][MC];
+        float mx[MR];
+#pragma unroll
+        for (int a = 0; a < MR; ++a) {
+            const int row = lr * MR + (a ^ gr);
+            float m = 0.f;
+#pragma unroll
+            for (int b = 0; b < MC; ++b) {
+                const int col = blk * M + lc * MC + (b ^ gc);
+                t[a][b] = sm.w[row * G::WS + col];
+                m = fmaxf(m, t[a][b]);
+            }
+            mx[a] = m;
+        }
+        if (P.iters > 0) {
+            reduce_scatter<MR, PC>(mx, 1, OpMax());
+            all_gather<MR, PC>(mx, 1);
+#pragma unroll
+            for (int a = 0; a < MR; ++a) {
+                const float sh = mx[a] * P.c_hi;
+#pragma unroll
+                for (int b = 0; b < MC; ++b) t[a][b] = fmaf(t[a][b], P.c_lo, fmaf(t[a][b], P.c_hi, -sh));
+            }
+            dykstra_iterate<M>(t, g, P.Nf, P.log2N, P.iters);
+#pragma unroll
+            for (int a = 0; a < MR; ++a)
+#pragma unroll
+                for (int b = 0; b < MC; ++b) t[a][b] = fminf(t[a][b], 0.0f);   // x = min(x + q, 0)
+        } else {
+#pragma unroll
+            for (int a = 0; a < MR; ++a)
+#pragma unroll
+                for (int b = 0; b < MC; ++b) t[a][b] = fmaf(t[a][b], P.c_lo, t[a][b] * P.c_hi);
+        }
+        if (MODE == 1) {
+            if (active) {
+#pragma unroll
+                for (int a = 0; a < MR; ++a)
+#pragma unroll
+                    for (int b = 0; b < MC; ++b) {
+                        const int64_t row = r0 + lr * MR + (a ^ gr);
+                        const int64_t col = c0 + blk * M + lc * MC + (b ^ gc);
+                        P.plan[row * P.ld_plan + col] = P.plan_is_log ? t[a][b] * 0.6931471805599453f : exp2f(t[a][b]);
+                    }
+            }
+        } else {
+#pragma unroll
+            for (int a = 0; a < MR; ++a)
+#pragma unroll
+                for (int b = 0; b < MC; ++b)
+                    sm.k[(lr * MR + (a ^ gr)) * G::WS + blk * M + lc * MC + (b ^ gc)] = t[a][b];
+        }
+        __syncwarp();
+    }
+
+    // ---- Algorithm 2 and the mask writer
+    if (MODE != 1) {
+        const int grp = lane / M;
+        RoundTables<M>& tb = sm.tb[warp * G::GPW + grp];
+#pragma unroll 1
+        for (int pass = 0; pass < G::PASSES; ++pass) {
+            const int blk = warp * G::BPW + pass * G::GPW + grp;
+            const bool active = blk * M < valid_cols;
+            const unsigned row_bits =
+                round_block<M>(sm.k + blk * M, sm.w + blk * M, tb, lane, active, P.N, P.ls_steps, flags);
+            if (active) {
+                const int off = blk * M;
+                if (M == 32) sm.bits[(lane % M) * G::WORDS + off / 32] = row_bits;
+                else atomicOr(&sm.bits[(lane % M) * G::WORDS + off / 32], row_bits << (off % 32));
+            }
+            __syncwarp();
+        }
+        __syncthreads();
+        const int nwords = (valid_cols + 31) / 32;
+        for (int idx = threadIdx.x; idx < M * G::WORDS; idx += WARPS * 32) {
+            const int r = idx / G::WORDS, wd = idx % G::WORDS;
+            if (wd < nwords) P.bits[(r0 + r) * P.wpr + c0 / 32 + wd] = sm.bits[idx];
+        }
+    }
+    flags = __reduce_or_sync(FULL, flags);
+    if (flags && lane == 0 && P.status) atomicOr(P.status, flags);
+}
+
+}  // namespace tsenor

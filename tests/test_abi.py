@@ -1,0 +1,62 @@
+"""CPU-side checks of the boundary: the C-ABI library builds for sm_100a, loads, exports
+every symbol that include/tsenor.h declares, and rejects bad arguments on the host
+(no kernel is launched here)."""
+import os
+import re
+
+import pytest
+
+from paper_2505_23949_b200 import binding as ts
+from paper_2505_23949_b200 import build as ts_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    ts_build.build()
+    return ts.lib()
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "tsenor.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return set(re.findall(r"\b(tsenor_[a-z_0-9]+)\s*\(", text))
+
+
+def test_library_exports_every_declared_symbol(lib):
+    declared = _declared_functions()
+    assert declared == set(ts.EXPORTS)
+    for name in declared:
+        assert getattr(lib, name) is not None
+
+
+def test_host_arithmetic_and_messages(lib):
+    assert [lib.tsenor_mask_words_per_row(c) for c in (0, 1, 32, 33, 4096)] == [0, 1, 1, 2, 128]
+    for code in (0, -1, -2, -3, -4, -5):
+        assert len(lib.tsenor_strerror(code)) > 1
+    assert lib.tsenor_strerror(-99) == b"unknown status"
+
+
+def test_argument_errors_are_decided_on_the_host(lib):
+    n0 = lib.tsenor_launch_count()
+    assert lib.tsenor_solve(None, 8, 8, 8, 2, 5, 1.0, 1, -1, None, None, None) == ts.ERR_NM
+    assert lib.tsenor_solve(None, 8, 8, 8, 5, 4, 1.0, 1, -1, None, None, None) == ts.ERR_NM
+    assert lib.tsenor_solve(None, 6, 8, 8, 2, 4, 1.0, 1, -1, None, None, None) == ts.ERR_SHAPE
+    assert lib.tsenor_solve(None, 8, 8, 4, 2, 4, 1.0, 1, -1, None, None, None) == ts.ERR_SHAPE
+    assert lib.tsenor_solve(None, 8, 8, 8, 2, 4, 1.0, -1, -1, None, None, None) == ts.ERR_ARG
+    assert lib.tsenor_solve(None, 8, 8, 8, 2, 4, 1.0, 1, -1, None, None, None) == ts.ERR_NULL
+    assert lib.tsenor_solve(None, 0, 8, 8, 2, 4, 1.0, 1, -1, None, None, None) == ts.OK
+    assert lib.tsenor_dykstra(None, 8, 8, 8, 4, 4, 1.0, 1, None, 8, 0, None, None) == ts.ERR_NM
+    assert lib.tsenor_dykstra(None, 8, 8, 8, 2, 4, 1.0, 1, None, 4, 0, None, None) == ts.ERR_SHAPE
+    assert lib.tsenor_round(None, 8, None, 8, 8, 8, 2, 4, -1, None, None, None) == ts.ERR_NULL
+    assert lib.tsenor_check(None, 8, 8, 2, 4, None, None) == ts.ERR_NULL
+    assert lib.tsenor_objective(None, 8, None, 8, 8, None, None) == ts.ERR_NULL
+    assert lib.tsenor_max_abs(None, 8, 8, 4, None, None) == ts.ERR_SHAPE
+    assert lib.tsenor_launch_count() == n0
+
+
+def test_binding_refuses_cpu_tensors(lib):
+    import torch
+    with pytest.raises(TypeError):
+        ts.solve(torch.zeros(8, 8), 2, 4, 1.0)

@@ -1,0 +1,236 @@
+"""GPU parity: the CUDA path, called through the C ABI (ctypes binding), against the
+CPU oracle on the same seeded inputs.  Tolerances are the ones the task states:
+plan within 1e-4 max-abs, rounding bit-exact on identical fp32 keys and scores, every
+block feasible, per-matrix objective within 1e-4 relative."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2505_23949_b200 import binding as ts
+from paper_2505_23949_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+PLAN_TOL = 1e-4
+OBJ_RTOL = 1e-4
+DEV = "cuda:0"
+
+# (M, N, rows, cols): several panels of the kernel's tiling plus a ragged last panel
+SHAPES = [
+    (4, 2, 24, 512 * 2 + 36),
+    (8, 4, 32, 512 * 2 + 72),
+    (16, 8, 48, 256 * 2 + 80),
+    (32, 16, 96, 128 * 2 + 96),
+    (8, 3, 16, 520),
+    (16, 5, 32, 272),
+    (32, 7, 64, 160),
+    (4, 1, 8, 516),
+    (4, 3, 8, 516),
+]
+
+
+def _scores(kind, rows, cols, seed):
+    if kind == "gauss":
+        return synth.gaussian_abs(rows, cols, 0.02, seed)
+    if kind == "student":
+        return synth.student_t_abs(rows, cols, 0.02, seed)
+    if kind == "wanda":
+        return synth.wanda_scores(rows, cols, 0.02, seed)
+    if kind == "outlier":
+        return synth.gaussian_outlier_columns_abs(rows, cols, 0.02, seed, frac=0.02)
+    raise ValueError(kind)
+
+
+def _dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
+
+
+def _bits(t):
+    return t.cpu().numpy().view(np.uint32)
+
+
+@pytest.mark.parametrize("kind", ["gauss", "student", "wanda", "outlier"])
+@pytest.mark.parametrize("M,N,rows,cols", SHAPES)
+def test_dykstra_plan_matches_oracle(kind, M, N, rows, cols):
+    W = _scores(kind, rows, cols, 17 * M + N)
+    tau = synth.default_tau(W.max())
+    st = ts.new_status(DEV)
+    plan = ts.dykstra(_dev(W), N, M, tau, 300, status=st).cpu().numpy()
+    ref = oracle.dykstra(W, N, M, tau, 300)
+    assert int(st.item()) == 0
+    err = np.abs(plan.astype(np.float64) - ref).max()
+    assert err <= PLAN_TOL, f"max|S_gpu - S_oracle| = {err:.3e}"
+    assert plan.max() <= 1.0 and plan.min() >= 0.0
+
+
+@pytest.mark.parametrize("iters", [0, 1, 2, 3, 17])
+def test_dykstra_few_iterations_and_log_plan(iters):
+    M, N = 16, 8
+    W = _scores("student", 32, 288, 5)
+    tau = synth.default_tau(W.max())
+    x = ts.dykstra(_dev(W), N, M, tau, iters, plan_is_log=True).cpu().numpy()
+    ref = oracle.dykstra(W, N, M, tau, iters, plan_is_log=True)
+    if iters == 0:
+        assert np.allclose(x, ref, rtol=2e-6, atol=1e-6)
+    else:
+        # compare where the plan is not negligible: log-plan differences there are relative errors of S
+        big = ref > -12
+        assert np.abs(x[big] - ref[big]).max() <= 2e-4
+        assert np.abs(np.exp(x.astype(np.float64)) - np.exp(ref)).max() <= PLAN_TOL
+
+
+def test_dykstra_literal_small_tau_and_tau_zero():
+    M, N = 8, 4
+    W = _scores("gauss", 16, 64, 9)
+    for tau in (0.0, 0.005 * float(W.max())):
+        plan = ts.dykstra(_dev(W), N, M, tau, 300).cpu().numpy()
+        ref = oracle.dykstra(W, N, M, tau, 300)
+        assert np.abs(plan - ref).max() <= 1e-5
+
+
+@pytest.mark.parametrize("keykind", ["plan", "ties", "cap", "scores"])
+@pytest.mark.parametrize("M,N,rows,cols", SHAPES)
+def test_rounding_is_bit_exact(keykind, M, N, rows, cols):
+    rng = np.random.default_rng(1000 * M + N)
+    W = _scores("wanda" if keykind == "ties" else "gauss", rows, cols, 31 * M + N)
+    if keykind == "plan":      # the log-plan the GPU itself produced (fp32)
+        key = ts.dykstra(_dev(W), N, M, synth.default_tau(W.max()), 300, plan_is_log=True).cpu().numpy()
+    elif keykind == "ties":    # few distinct values: the index tie-break decides almost everything
+        key = np.round(rng.standard_normal((rows, cols)) * 1.5).astype(np.float32)
+        key[::3, ::5] = -0.0
+        key[1::3, ::7] = 0.0
+    elif keykind == "cap":     # many entries exactly at the cap (x = 0), as after the clip
+        key = np.minimum(rng.standard_normal((rows, cols)), 0).astype(np.float32)
+    else:                      # Algorithm 2 applied to |W| itself
+        key = W.copy()
+    for ls in (-1, 0, 1, 10):
+        st = ts.new_status(DEV)
+        got = _bits(ts.round_plan(_dev(key), _dev(W), N, M, ls_steps=ls, status=st))
+        want, info = oracle.round_plan(key, W, N, M, ls_steps=ls, stats=True)
+        assert np.array_equal(got, want), f"ls_steps={ls}: {np.count_nonzero(got != want)} words differ"
+        flags = int(st.item())
+        assert (flags & ts.DEV_INTERNAL) == 0 and (flags & ts.DEV_NONFINITE_SCORE) == 0
+        assert bool(flags & ts.DEV_UNDERFILLED) == (info["underfilled"] > 0)
+        if ls < 0:
+            assert oracle.count_infeasible(got, rows, cols, N, M) == 0
+
+
+@pytest.mark.parametrize("kind", ["gauss", "student", "wanda", "outlier"])
+@pytest.mark.parametrize("M,N,rows,cols", SHAPES)
+def test_solve_feasible_and_objective_matches_oracle(kind, M, N, rows, cols):
+    W = _scores(kind, rows, cols, 53 * M + N)
+    tau = synth.default_tau(W.max())
+    Wd = _dev(W)
+    st = ts.new_status(DEV)
+    mask = ts.solve(Wd, N, M, tau, 300, status=st)
+    got = _bits(mask)
+    assert int(st.item()) == 0
+    assert oracle.count_infeasible(got, rows, cols, N, M) == 0
+    assert int(ts.check(mask, rows, cols, N, M).item()) == 0
+    want = oracle.solve(W, N, M, tau, 300)
+    o_gpu, o_ref = oracle.objective(W, got), oracle.objective(W, want)
+    assert abs(o_gpu - o_ref) <= OBJ_RTOL * o_ref
+    # the library's own objective reduction agrees with the oracle's on the same mask
+    assert abs(float(ts.objective(Wd, mask).item()) - o_gpu) <= 1e-9 * o_gpu
+    # fused kernel == stage kernels chained (same arithmetic, same tie-breaks)
+    key = ts.dykstra(Wd, N, M, tau, 300, plan_is_log=True)
+    assert np.array_equal(_bits(ts.round_plan(key, Wd, N, M)), got)
+
+
+def test_solve_config1_full_and_brute_force_2_4():
+    wl = synth.config(1)
+    tau = synth.default_tau(wl.scores.max())
+    got = _bits(ts.solve(_dev(wl.scores), wl.N, wl.M, tau, 300))
+    assert oracle.count_infeasible(got, 512, 512, wl.N, wl.M) == 0
+    want = oracle.solve(wl.scores, wl.N, wl.M, tau, 300)
+    o_gpu, o_ref = oracle.objective(wl.scores, got), oracle.objective(wl.scores, want)
+    assert abs(o_gpu - o_ref) <= OBJ_RTOL * o_ref
+    # 2:4: every block's objective against the optimum over all 90 feasible masks
+    W = synth.gaussian_abs(256, 1024, 0.02, 2000)
+    got = _bits(ts.solve(_dev(W), 2, 4, synth.default_tau(W.max()), 300))
+    opt = oracle.bruteforce(W, 2, 4)
+    obj = oracle.block_objectives(W, got, 4)
+    assert np.all(obj <= opt + 1e-9)
+    assert np.mean(obj >= opt - 1e-9) > 0.98
+
+
+def test_strided_and_unaligned_inputs():
+    M, N = 8, 4
+    rng = np.random.default_rng(3)
+    big = np.abs(rng.standard_normal((40, 300))).astype(np.float32)
+    bigd = _dev(big)
+    for r0, c0, rows, cols in [(0, 0, 32, 288), (1, 3, 32, 264), (8, 4, 16, 40)]:
+        view = bigd[r0:r0 + rows, c0:c0 + cols]            # ld = 300, base maybe unaligned
+        W = big[r0:r0 + rows, c0:c0 + cols].copy()
+        tau = synth.default_tau(W.max())
+        got = _bits(ts.solve(view, N, M, tau, 50))
+        ref = _bits(ts.solve(_dev(W), N, M, tau, 50))
+        assert np.array_equal(got, ref)
+        assert oracle.count_infeasible(got, rows, cols, N, M) == 0
+        planv = torch.zeros((rows, 310), device=DEV)[:, 5:5 + cols]
+        ts.dykstra(view, N, M, tau, 50, plan_out=planv)
+        assert np.abs(planv.cpu().numpy() - oracle.dykstra(W, N, M, tau, 50)).max() <= PLAN_TOL
+
+
+def test_trivial_patterns_empty_inputs_and_helpers():
+    W = _scores("gauss", 16, 72, 1)
+    Wd = _dev(W)
+    zero = _bits(ts.solve(Wd, 0, 8, 1.0, 10))
+    ones = _bits(ts.solve(Wd, 8, 8, 1.0, 10))
+    assert not zero.any()
+    dense = oracle.unpack_mask(ones, 72)
+    assert dense.all() and ones[:, 2].max() == 0xFF          # bits past column 71 stay 0
+    assert ts.solve(torch.empty((0, 64), device=DEV), 4, 8, 1.0, 10).shape == (0, 2)
+    assert abs(float(ts.max_abs(Wd).item()) - float(W.max())) == 0.0
+    assert float(ts.max_abs(-Wd).item()) == float(W.max())
+    m = ts.solve(Wd, 4, 8, synth.default_tau(W.max()), 300)
+    assert int(ts.check(m, 16, 72, 4, 8).item()) == 0
+    bad = m.clone()
+    bad[0, 0] ^= 1
+    bad[9, 1] ^= 4
+    assert int(ts.check(bad, 16, 72, 4, 8).item()) == 2
+    assert int(ts.check(m, 16, 72, 3, 8).item()) == 2 * 9
+
+
+def test_host_side_errors_do_not_launch():
+    W = _dev(_scores("gauss", 16, 64, 2))
+    n0 = ts.launch_count()
+    for kwargs, code in [
+        (dict(N=4, M=6), ts.ERR_NM), (dict(N=9, M=8), ts.ERR_NM), (dict(N=-1, M=8), ts.ERR_NM),
+        (dict(N=4, M=8, iters=-1), ts.ERR_ARG), (dict(N=4, M=8, tau=float("nan")), ts.ERR_ARG),
+        (dict(N=4, M=8, tau=-1.0), ts.ERR_ARG), (dict(N=16, M=32), ts.ERR_SHAPE),
+    ]:
+        args = dict(N=4, M=8, tau=1.0, iters=5)
+        args.update(kwargs)
+        with pytest.raises(ts.TsenorError) as e:
+            ts.solve(W, **args)
+        assert e.value.status == code
+    with pytest.raises(ts.TsenorError) as e:
+        ts.dykstra(W, 8, 8, 1.0, 5)
+    assert e.value.status == ts.ERR_NM
+    rc = ts.lib().tsenor_solve(None, 16, 64, 64, 4, 8, 1.0, 5, -1, None, None, None)
+    assert rc == ts.ERR_NULL
+    assert ts.launch_count() == n0
+
+
+def test_non_finite_scores_are_flagged_and_nothing_hangs():
+    M, N = 8, 4
+    W = _scores("gauss", 16, 128, 4)
+    W[3, 5] = np.nan
+    W[9, 70] = np.inf
+    st = ts.new_status(DEV)
+    mask = ts.solve(_dev(W), N, M, 100.0, 300, status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) & ts.DEV_NONFINITE_SCORE
+    got = _bits(mask)
+    # blocks without a planted value are unaffected
+    clean = W.copy()
+    clean[3, 5] = 0
+    clean[9, 70] = 0
+    ref = _bits(ts.solve(_dev(clean), N, M, 100.0, 300))
+    keep = np.ones_like(got, bool)
+    keep[0:8, 0] = False      # block (0,0) holds the NaN  -> word 0 rows 0..7, bits 0..7
+    keep[8:16, 2] = False     # block (1,8) holds the inf  -> word 2 rows 8..15
+    assert np.array_equal(got[keep], ref[keep])
+    assert np.array_equal(got[0:8, 0] >> 8, ref[0:8, 0] >> 8)
