@@ -43,7 +43,7 @@ int launch(const tsenor::Params& P, cudaStream_t st) {
     if (panels > 0x7fffffffLL) return TSENOR_ERR_SHAPE;
     tsenor::Params Q = P;
     Q.npc = (int)npc;
-    const size_t smem = sizeof(tsenor::SmemLayout<M>);
+    const size_t smem = sizeof(tsenor::SmemLayout<M, MODE>);
     static thread_local int configured_device = -1;
     int dev = 0;
     cudaGetDevice(&dev);

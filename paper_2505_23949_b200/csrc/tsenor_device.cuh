@@ -181,17 +181,30 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>:
         }
         all_gather<MC, PR>(G, PC);
     }
+    // Steady state.  Element-wise work runs on pairs of columns with the packed
+    // fp32x2 add / fma of sm_100, which halves its issue slots; exp2 and the clip
+    // stay scalar.
+    constexpr int MP = MC / 2;
+    float2 tp[MR][MP];
+#pragma unroll
+    for (int a = 0; a < MR; ++a)
+#pragma unroll
+        for (int b = 0; b < MP; ++b) tp[a][b] = make_float2(t[a][2 * b], t[a][2 * b + 1]);
     for (int it = 1; it < iters; ++it) {
-        float e[MR][MC], rp[MR], rho[MR], cp[MC];
+        float2 e[MR][MP], cp2[MP];
+        float rp[MR], rho[MR], cp[MC];
 #pragma unroll
         for (int a = 0; a < MR; ++a) {
-            float s = 0.f;
+            const float2 Fa = make_float2(F[a], F[a]);
+            float2 s2;
 #pragma unroll
-            for (int b = 0; b < MC; ++b) {
-                e[a][b] = fminf(ex2_approx((t[a][b] + F[a]) + G[b]), 1.0f);
-                s += e[a][b];
+            for (int b = 0; b < MP; ++b) {
+                const float2 arg = __fadd2_rn(__fadd2_rn(tp[a][b], Fa), make_float2(G[2 * b], G[2 * b + 1]));
+                e[a][b].x = fminf(ex2_approx(arg.x), 1.0f);
+                e[a][b].y = fminf(ex2_approx(arg.y), 1.0f);
+                s2 = (b == 0) ? e[a][b] : __fadd2_rn(s2, e[a][b]);
             }
-            rp[a] = s;
+            rp[a] = s2.x + s2.y;
         }
         reduce_scatter<MR, PC>(rp, 1, OpAdd());
 #pragma unroll
@@ -203,11 +216,12 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>:
         all_gather<MR, PC>(rho, 1);
         all_gather<MR, PC>(F, 1);
 #pragma unroll
-        for (int b = 0; b < MC; ++b) {
-            float s = e[0][b] * rho[0];
+        for (int b = 0; b < MP; ++b) {
+            cp2[b] = __fmul2_rn(e[0][b], make_float2(rho[0], rho[0]));
 #pragma unroll
-            for (int a = 1; a < MR; ++a) s = fmaf(e[a][b], rho[a], s);
-            cp[b] = s;
+            for (int a = 1; a < MR; ++a) cp2[b] = __ffma2_rn(e[a][b], make_float2(rho[a], rho[a]), cp2[b]);
+            cp[2 * b] = cp2[b].x;
+            cp[2 * b + 1] = cp2[b].y;
         }
         reduce_scatter<MC, PR>(cp, PC, OpAdd());
 #pragma unroll
@@ -473,21 +487,31 @@ struct Params {
     int vec_scores, vec_keys;
 };
 
-template <int M> struct SmemLayout {
+template <int M, int MODE> struct SmemLayout {
     using G = Geom<M>;
     float w[M * G::WS];
     float k[M * G::WS];
     RoundTables<M> tb[WARPS * G::GPW];
     unsigned int bits[M * G::WORDS];
 };
+template <int M> struct SmemLayout<M, 1> {   // Algorithm 1 alone needs the score panel only
+    using G = Geom<M>;
+    float w[M * G::WS];
+    float k[1];
+    RoundTables<M> tb[1];
+    unsigned int bits[1];
+};
+#ifndef TSENOR_MINB
+#define TSENOR_MINB 1
+#endif
 
 template <int M, int MODE>
-__global__ void __launch_bounds__(WARPS * 32) tsenor_kernel(const Params P) {
+__global__ void __launch_bounds__(WARPS * 32, TSENOR_MINB) tsenor_kernel(const Params P) {
     using G = Geom<M>;
     using T = Tile<M>;
     constexpr int MR = T::MR, MC = T::MC, PR = T::PR, PC = T::PC;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    SmemLayout<M>& sm = *reinterpret_cast<SmemLayout<M>*>(smem_raw);
+    SmemLayout<M, MODE>& sm = *reinterpret_cast<SmemLayout<M, MODE>*>(smem_raw);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t panel = blockIdx.x;
