@@ -38,7 +38,6 @@ template <int M> struct Geom {
     static constexpr int WS = PANEL + 1;             // shared row stride (floats)
     static constexpr int GPW = 32 / M;               // rounding groups per warp
     static constexpr int PASSES = BPW / GPW;         // rounding passes per warp
-    static constexpr int TS = M + 4;                 // byte-table row stride
     static constexpr int WORDS = PANEL / 32;         // mask words per panel row
 };
 
@@ -109,35 +108,53 @@ struct Comp {
 };
 
 // ---------------------------------------------------------------------------
-// Algorithm 1 in potential form.
+// Algorithm 1 in potential form, with stabilised linear-domain steps.
 //
 // In the log domain the three projections only ever add a row term and a
 // column term to x + q, and after the clip x = min(t, 0), q = max(t, 0) for
 // t = x + q.  So the whole state is t_ij = t0_ij + F_i + G_j with
-// t0 = tau |w| (base-2 units here), and one iteration is
-//     e_ij   = min(2^t_ij, 1)                      (S of the previous clip)
-//     F_i   += log2 N - log2 sum_j e_ij            (projection on C1)
-//     G_j   += log2 N - log2 sum_i e_ij N / r_i    (projection on C2)
-// with the clip (C3) and the dual update implicit in the next e.  One exp per
-// element and iteration.  Iteration 0 has no clip yet and its column pass is
-// done with the maximum subtracted, because 2^t0 of a whole column can
-// underflow against a large entry elsewhere in its rows; from iteration 1 on
-// every row and column sum is bounded below by N/M, so no sum can vanish.
+// t0 = tau |w| (base-2 units here), and with U = 2^t (the unclipped S .* Q)
+// one iteration is
+//     e_ij   = min(U_ij, 1)                        (S after the previous clip)
+//     rho_i  = N / sum_j e_ij                      (projection on C1)
+//     kap_j  = N / sum_i e_ij rho_i                (projection on C2)
+//     U_ij  <- U_ij rho_i kap_j ,  F_i += log2 rho_i ,  G_j += log2 kap_j
+// with the clip (C3) and the dual update implicit in the next e.  U is the
+// linear-domain iterate of Algorithm 1; it is only trusted for RESYNC
+// iterations at a time and then rebuilt as 2^(t0 + F + G) from the log-domain
+// potentials, which is what keeps large tau |w| safe in fp32: an entry that
+// overflowed stays clipped and one that flushed to zero stays negligible for
+// that long, because from iteration 1 on every rho*kap lies in
+// [N/M^3, N M^2] (row sums of e are in [1/M, M], column sums of e*rho in
+// [N/M, N M^2]).  Iteration 0 has no clip yet and is done entirely in the
+// log domain with the column maximum subtracted, because 2^t0 of a whole
+// column can underflow against a large entry elsewhere in its rows.
+//
 // On entry t holds t0 with its row maximum subtracted (exact no-op for the
 // method: the first row projection removes any row constant); on return t
-// holds the final t = x + q.
+// holds the final t = x + q.  stash: 32 * MR * MC floats of shared memory
+// private to the warp (keeps t0 while the registers hold U).
 // ---------------------------------------------------------------------------
+constexpr int RESYNC = 6;   // (N M^2)^6 < 2^90: a flushed entry stays below 2^-36
+
 template <int M>
-__device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>::MC], int lane_in_blk,
+__device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>::MC], float* stash, int lane,
                                                 float Nf, float log2N, int iters) {
     using T = Tile<M>;
     constexpr int MR = T::MR, MC = T::MC, PR = T::PR, PC = T::PC;
     constexpr int RO = MR / PC, CO = MC / PR;  // lines whose sums this lane finishes
-    (void)lane_in_blk;
+    constexpr int MP = MC / 2, NQ = MR * MC / 4;
     float F[MR], G[MC];
     Comp Fo[RO], Go[CO];
+    float Pr[RO], Pc[CO];                      // products of rho / kap since the last resync
     if (iters <= 0) return;
-    {   // iteration 0
+    float4* const st4 = reinterpret_cast<float4*>(stash) + lane;
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) {
+        const int a = (4 * q) / MC, b = (4 * q) % MC;
+        st4[q * 32] = make_float4(t[a][b], t[a][b + 1], t[a][b + 2], t[a][b + 3]);
+    }
+    {   // iteration 0, log domain
         float rp[MR];
 #pragma unroll
         for (int a = 0; a < MR; ++a) {
@@ -152,6 +169,7 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>:
             Fo[k].hi = log2N - lg2_approx(rp[k]);
             Fo[k].lo = 0.f;
             F[k] = Fo[k].hi;
+            Pr[k] = 1.0f;
         }
         all_gather<MR, PC>(F, 1);
         float cm[MC];
@@ -177,31 +195,43 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>:
         for (int k = 0; k < CO; ++k) {
             Go[k].hi = (log2N - cm[k]) - lg2_approx(cp[k]);
             Go[k].lo = 0.f;
-            G[k] = Go[k].hi;
+            Pc[k] = 1.0f;
         }
-        all_gather<MC, PR>(G, PC);
     }
-    // Steady state.  Element-wise work runs on pairs of columns with the packed
-    // fp32x2 add / fma of sm_100, which halves its issue slots; exp2 and the clip
-    // stay scalar.
-    constexpr int MP = MC / 2;
-    float2 tp[MR][MP];
-#pragma unroll
-    for (int a = 0; a < MR; ++a)
-#pragma unroll
-        for (int b = 0; b < MP; ++b) tp[a][b] = make_float2(t[a][2 * b], t[a][2 * b + 1]);
+    // Iterations 1 .. iters-1.  Element-wise work runs on pairs of columns with
+    // the packed fp32x2 add / mul / fma of sm_100 (half the issue slots).
+    float2 U[MR][MP];
+    int until_resync = 0;
     for (int it = 1; it < iters; ++it) {
-        float2 e[MR][MP], cp2[MP];
-        float rp[MR], rho[MR], cp[MC];
+        if (until_resync == 0) {
+            until_resync = RESYNC;
+#pragma unroll
+            for (int k = 0; k < RO; ++k) { Fo[k].add(lg2_approx(Pr[k])); Pr[k] = 1.0f; F[k] = Fo[k].hi; }
+#pragma unroll
+            for (int k = 0; k < CO; ++k) { Go[k].add(lg2_approx(Pc[k])); Pc[k] = 1.0f; G[k] = Go[k].hi; }
+            all_gather<MR, PC>(F, 1);
+            all_gather<MC, PR>(G, PC);
+#pragma unroll
+            for (int q = 0; q < NQ; ++q) {
+                const int a = (4 * q) / MC, b = ((4 * q) % MC) / 2;
+                const float4 v = st4[q * 32];
+                const float2 Fa = make_float2(F[a], F[a]);
+                const float2 x0 = __fadd2_rn(__fadd2_rn(make_float2(v.x, v.y), Fa), make_float2(G[2 * b], G[2 * b + 1]));
+                const float2 x1 =
+                    __fadd2_rn(__fadd2_rn(make_float2(v.z, v.w), Fa), make_float2(G[2 * b + 2], G[2 * b + 3]));
+                U[a][b] = make_float2(ex2_approx(x0.x), ex2_approx(x0.y));
+                U[a][b + 1] = make_float2(ex2_approx(x1.x), ex2_approx(x1.y));
+            }
+        }
+        --until_resync;
+        float2 e[MR][MP];
+        float rp[MR], rho[MR], cp[MC], kap[MC];
 #pragma unroll
         for (int a = 0; a < MR; ++a) {
-            const float2 Fa = make_float2(F[a], F[a]);
             float2 s2;
 #pragma unroll
             for (int b = 0; b < MP; ++b) {
-                const float2 arg = __fadd2_rn(__fadd2_rn(tp[a][b], Fa), make_float2(G[2 * b], G[2 * b + 1]));
-                e[a][b].x = fminf(ex2_approx(arg.x), 1.0f);
-                e[a][b].y = fminf(ex2_approx(arg.y), 1.0f);
+                e[a][b] = make_float2(fminf(U[a][b].x, 1.0f), fminf(U[a][b].y, 1.0f));
                 s2 = (b == 0) ? e[a][b] : __fadd2_rn(s2, e[a][b]);
             }
             rp[a] = s2.x + s2.y;
@@ -210,31 +240,48 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>:
 #pragma unroll
         for (int k = 0; k < RO; ++k) {
             rho[k] = Nf * rcp_approx(rp[k]);
-            Fo[k].add(log2N - lg2_approx(rp[k]));
-            F[k] = Fo[k].hi;
+            Pr[k] *= rho[k];
         }
         all_gather<MR, PC>(rho, 1);
-        all_gather<MR, PC>(F, 1);
 #pragma unroll
         for (int b = 0; b < MP; ++b) {
-            cp2[b] = __fmul2_rn(e[0][b], make_float2(rho[0], rho[0]));
+            float2 c2 = __fmul2_rn(e[0][b], make_float2(rho[0], rho[0]));
 #pragma unroll
-            for (int a = 1; a < MR; ++a) cp2[b] = __ffma2_rn(e[a][b], make_float2(rho[a], rho[a]), cp2[b]);
-            cp[2 * b] = cp2[b].x;
-            cp[2 * b + 1] = cp2[b].y;
+            for (int a = 1; a < MR; ++a) c2 = __ffma2_rn(e[a][b], make_float2(rho[a], rho[a]), c2);
+            cp[2 * b] = c2.x;
+            cp[2 * b + 1] = c2.y;
         }
         reduce_scatter<MC, PR>(cp, PC, OpAdd());
 #pragma unroll
         for (int k = 0; k < CO; ++k) {
-            Go[k].add(log2N - lg2_approx(cp[k]));
-            G[k] = Go[k].hi;
+            kap[k] = Nf * rcp_approx(cp[k]);
+            Pc[k] *= kap[k];
         }
-        all_gather<MC, PR>(G, PC);
+        all_gather<MC, PR>(kap, PC);
+#pragma unroll
+        for (int a = 0; a < MR; ++a) {
+            const float2 ra = make_float2(rho[a], rho[a]);
+#pragma unroll
+            for (int b = 0; b < MP; ++b)
+                U[a][b] = __fmul2_rn(__fmul2_rn(U[a][b], ra), make_float2(kap[2 * b], kap[2 * b + 1]));
+        }
     }
+    // final potentials and t = t0 + F + G
 #pragma unroll
-    for (int a = 0; a < MR; ++a)
+    for (int k = 0; k < RO; ++k) { Fo[k].add(lg2_approx(Pr[k])); F[k] = Fo[k].hi; }
 #pragma unroll
-        for (int b = 0; b < MC; ++b) t[a][b] = (t[a][b] + F[a]) + G[b];
+    for (int k = 0; k < CO; ++k) { Go[k].add(lg2_approx(Pc[k])); G[k] = Go[k].hi; }
+    all_gather<MR, PC>(F, 1);
+    all_gather<MC, PR>(G, PC);
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) {
+        const int a = (4 * q) / MC, b = (4 * q) % MC;
+        const float4 v = st4[q * 32];
+        t[a][b] = (v.x + F[a]) + G[b];
+        t[a][b + 1] = (v.y + F[a]) + G[b + 1];
+        t[a][b + 2] = (v.z + F[a]) + G[b + 2];
+        t[a][b + 3] = (v.w + F[a]) + G[b + 3];
+    }
 }
 
 // ---------------------------------------------------------------------------
@@ -273,12 +320,15 @@ __device__ __forceinline__ int load_panel(const float* __restrict__ src, int64_t
 // Rounding stage (Algorithm 2).  A group of M lanes owns one block; lane i of
 // the group plays row i and column i at once.
 // ---------------------------------------------------------------------------
-template <int M> struct RoundTables {
-    static constexpr int TS = Geom<M>::TS;
-    unsigned char rperm[M * TS];  // [i][p] -> column of the p-th best entry of row i
-    unsigned char cperm[M * TS];  // [j][s] -> row of the s-th best entry of column j
-    unsigned char rrank[M * TS];  // [i][j] -> rank of (i,j) inside row i
-    unsigned char crank[M * TS];  // [j][i] -> rank of (i,j) inside column j
+// Per-group scratch of the rounding stage.  The four byte tables that hold the
+// sorted orders (each lane only ever reads its own line of them) are written
+// over the block's own key cells once both sorts have consumed the keys: key
+// row i (M floats = 4M bytes) becomes
+//   [0,M)   rperm[p] -> column of the p-th best entry of row i
+//   [M,2M)  cperm[s] -> row of the s-th best entry of column i
+//   [2M,3M) rrank[j] -> rank of (i,j) inside row i
+//   [3M,4M) crank[r] -> rank of (r,i) inside column i
+template <int M> struct RoundScratch {
     unsigned int rs[M];           // row-side picks of the round, bits over columns
     unsigned int cs[M];           // column-side picks of the round, bits over rows
     unsigned int sel[M];          // current mask, one word per row
@@ -311,38 +361,54 @@ template <int M> __device__ __forceinline__ void sort_regs(unsigned long long (&
             }
 }
 
-// Sorts one line (stride `st` floats in shared memory) and writes the
-// permutation and rank tables for it.
+// Sorts one line (stride `st` floats in shared memory); returns the permutation
+// packed four indices per word (byte p%4 of word p/4 = index of the p-th best).
 template <int M>
-__device__ __forceinline__ void sort_line(const float* line, int st, unsigned char* perm, unsigned char* rank) {
+__device__ __forceinline__ void sort_line(const float* line, int st, unsigned (&packed)[M / 4]) {
     unsigned long long v[M];
 #pragma unroll
     for (int k = 0; k < M; ++k) v[k] = sort_word(line[k * st], k);
     sort_regs<M>(v);
 #pragma unroll
-    for (int p = 0; p < M; ++p) {
-        const int k = (int)(v[p] & 63u);
-        perm[p] = (unsigned char)k;
-        rank[k] = (unsigned char)p;
-    }
+    for (int w = 0; w < M / 4; ++w)
+        packed[w] = ((unsigned)v[4 * w] & 63u) | (((unsigned)v[4 * w + 1] & 63u) << 8) |
+                    (((unsigned)v[4 * w + 2] & 63u) << 16) | (((unsigned)v[4 * w + 3] & 63u) << 24);
+}
+template <int M>
+__device__ __forceinline__ void store_tables(const unsigned (&packed)[M / 4], unsigned char* perm, unsigned char* rank) {
+#pragma unroll
+    for (int w = 0; w < M / 4; ++w) reinterpret_cast<unsigned*>(perm)[w] = packed[w];
+#pragma unroll
+    for (int p = 0; p < M; ++p) rank[(packed[p / 4] >> (8 * (p % 4))) & 0xffu] = (unsigned char)p;
 }
 
 // Greedy selection + local search for the block of this lane's group.
 //   ks, ws: shared-memory pointers to element (0,0) of the block's keys and
-//   |scores| (row stride WS); tb: the group's tables; active: group has a block.
+//   |scores| (row stride WS); the key cells are overwritten.  tb: the group's
+//   scratch; active: group has a block.
 // Returns this lane's row of the mask (M bits).  flags accumulates DEV_* bits.
 template <int M>
-__device__ __forceinline__ unsigned round_block(const float* ks, const float* ws, RoundTables<M>& tb, int lane,
+__device__ __forceinline__ unsigned round_block(float* ks, const float* ws, RoundScratch<M>& tb, int lane,
                                                 bool active, int N, int ls_steps, int& flags) {
     using G = Geom<M>;
-    constexpr int WS = G::WS, TS = G::TS;
+    constexpr int WS = G::WS;
     constexpr unsigned GM = (M == 32) ? 0xffffffffu : ((1u << (M & 31)) - 1u);
     const int i = lane % M;            // my row, and my column
     const int gsh = (lane / M) * M;    // first lane of my group
 
     // ---- sorted orders of my row and of my column (Algorithm 2 line 2)
-    sort_line<M>(ks + i * WS, 1, tb.rperm + i * TS, tb.rrank + i * TS);
-    sort_line<M>(ks + i, WS, tb.cperm + i * TS, tb.crank + i * TS);
+    unsigned char* const rperm = reinterpret_cast<unsigned char*>(ks + i * WS);
+    unsigned char* const cperm = rperm + M;
+    unsigned char* const rrank = rperm + 2 * M;
+    unsigned char* const crank = rperm + 3 * M;
+    {
+        unsigned pr[M / 4], pc[M / 4];
+        sort_line<M>(ks + i * WS, 1, pr);
+        sort_line<M>(ks + i, WS, pc);
+        __syncwarp();                       // every lane is done reading keys
+        store_tables<M>(pr, rperm, rrank);
+        store_tables<M>(pc, cperm, crank);
+    }
     __syncwarp();
 
     // ---- greedy selection (lines 3-6) in synchronous rounds.  An available
@@ -367,13 +433,13 @@ __device__ __forceinline__ unsigned round_block(const float* ks, const float* ws
                 const int p = __ffs(ar) - 1;
                 ar &= ar - 1; --nr;
                 pickR |= 1u << p;
-                RS |= 1u << tb.rperm[i * TS + p];
+                RS |= 1u << rperm[p];
             }
             if (nc > 0 && bc) {
                 const int s = __ffs(bc) - 1;
                 bc &= bc - 1; --nc;
                 pickC |= 1u << s;
-                CS |= 1u << tb.cperm[i * TS + s];
+                CS |= 1u << cperm[s];
             }
         }
         tb.rs[i] = RS;
@@ -384,13 +450,13 @@ __device__ __forceinline__ unsigned round_block(const float* ks, const float* ws
             if (pickR) {
                 const int p = __ffs(pickR) - 1;
                 pickR &= pickR - 1;
-                const int j = tb.rperm[i * TS + p];
+                const int j = rperm[p];
                 if ((tb.cs[j] >> i) & 1u) { sel |= 1u << j; A &= ~(1u << p); --capR; }
             }
             if (pickC) {
                 const int s = __ffs(pickC) - 1;
                 pickC &= pickC - 1;
-                const int r = tb.cperm[i * TS + s];
+                const int r = cperm[s];
                 if ((tb.rs[r] >> i) & 1u) { B &= ~(1u << s); --capC; }
             }
         }
@@ -405,12 +471,12 @@ __device__ __forceinline__ unsigned round_block(const float* ks, const float* ws
             if (nfr) {
                 const int r = __ffs(nfr) - 1;
                 nfr &= nfr - 1;
-                B &= ~(1u << tb.crank[i * TS + r]);
+                B &= ~(1u << crank[r]);
             }
             if (nfc) {
                 const int c = __ffs(nfc) - 1;
                 nfc &= nfc - 1;
-                A &= ~(1u << tb.rrank[i * TS + c]);
+                A &= ~(1u << rrank[c]);
             }
         }
     }
@@ -491,22 +557,21 @@ template <int M, int MODE> struct SmemLayout {
     using G = Geom<M>;
     float w[M * G::WS];
     float k[M * G::WS];
-    RoundTables<M> tb[WARPS * G::GPW];
+    RoundScratch<M> tb[WARPS * G::GPW];
     unsigned int bits[M * G::WORDS];
 };
-template <int M> struct SmemLayout<M, 1> {   // Algorithm 1 alone needs the score panel only
+template <int M> struct SmemLayout<M, 1> {   // Algorithm 1 alone: score panel and the t0 stash
     using G = Geom<M>;
     float w[M * G::WS];
-    float k[1];
-    RoundTables<M> tb[1];
+    float k[WARPS * 32 * Tile<M>::MR * Tile<M>::MC];
+    RoundScratch<M> tb[1];
     unsigned int bits[1];
 };
-#ifndef TSENOR_MINB
-#define TSENOR_MINB 1
-#endif
+// Resident CTAs per SM the register allocation aims for.
+template <int M> struct MinBlocks { static constexpr int value = (M == 32 || M == 4) ? 5 : 4; };
 
 template <int M, int MODE>
-__global__ void __launch_bounds__(WARPS * 32, TSENOR_MINB) tsenor_kernel(const Params P) {
+__global__ void __launch_bounds__(WARPS * 32, MinBlocks<M>::value) tsenor_kernel(const Params P) {
     using G = Geom<M>;
     using T = Tile<M>;
     constexpr int MR = T::MR, MC = T::MC, PR = T::PR, PC = T::PC;
@@ -558,7 +623,7 @@ __global__ void __launch_bounds__(WARPS * 32, TSENOR_MINB) tsenor_kernel(const P
 #pragma unroll
                 for (int b = 0; b < MC; ++b) t[a][b] = fmaf(t[a][b], P.c_lo, fmaf(t[a][b], P.c_hi, -sh));
             }
-            dykstra_iterate<M>(t, g, P.Nf, P.log2N, P.iters);
+            dykstra_iterate<M>(t, sm.k + warp * (32 * MR * MC), lane, P.Nf, P.log2N, P.iters);
 #pragma unroll
             for (int a = 0; a < MR; ++a)
 #pragma unroll
@@ -581,6 +646,7 @@ __global__ void __launch_bounds__(WARPS * 32, TSENOR_MINB) tsenor_kernel(const P
                     }
             }
         } else {
+            __syncthreads();   // sm.k served as per-warp stash until here; now it takes the keys
 #pragma unroll
             for (int a = 0; a < MR; ++a)
 #pragma unroll
@@ -593,7 +659,7 @@ __global__ void __launch_bounds__(WARPS * 32, TSENOR_MINB) tsenor_kernel(const P
     // ---- Algorithm 2 and the mask writer
     if (MODE != 1) {
         const int grp = lane / M;
-        RoundTables<M>& tb = sm.tb[warp * G::GPW + grp];
+        RoundScratch<M>& tb = sm.tb[warp * G::GPW + grp];
 #pragma unroll 1
         for (int pass = 0; pass < G::PASSES; ++pass) {
             const int blk = warp * G::BPW + pass * G::GPW + grp;
