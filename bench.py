@@ -27,18 +27,29 @@ from paper_2505_23949_b200 import synth  # noqa: E402
 T_ITERS = 300
 LS_STEPS = -1
 SM_COUNT = 148
+FMA_LANES_PER_CLK_PER_SM = 128  # fp32 add/mul/fma lanes per clock per SM
 XU_PER_CLK_PER_SM = 16          # special-function results per clock per SM
 NOMINAL_SM_MHZ = 1965.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one tsenor_kernel<32,0> launch on the
+# 14336x4096 matrix, from the ncu capture summarised under profiles/ (None until captured)
+NCU_DRAM_BYTES_PER_LAUNCH = None
 
 
-def xu_ops_per_block(M, T):
-    """Special-function operations the kernel's algorithm needs per block: M^2 exp2 plus
-    2M log2 and M reciprocals per iteration (one exp per element and iteration)."""
+def fma_lane_ops_per_block(M, T):
+    """fp32 FMA-pipe lane operations one block needs in the kernel's formulation of
+    Algorithm 1: per element and iteration one row-sum add, one column-sum fma and the two
+    scalings by rho_i and kappa_j (the clip is a min on the integer/ALU pipe and the
+    exp2 resync every 6th iteration is on the SFU; neither is counted)."""
+    return 4 * M * M * T
+
+
+def xu_ops_per_block_one_exp(M, T):
+    """SFU operations of a log-domain iteration with one exp per element and iteration."""
     return (M * M + 3 * M) * T
 
 
 def xu_ops_per_block_literal(M, T):
-    """Same count for the paper's listing: two log-sum-exps per iteration."""
+    """SFU operations of the paper's listing: two log-sum-exps per iteration."""
     return (2 * M * M + 2 * M) * T
 
 
@@ -292,9 +303,12 @@ def run_cuda(args, rank, world, local_rank):
         value = world * blocks_per_step * args.steps / sec
         mean_launch_s = statistics.mean(launch_ms) / 1e3
         blocks_per_launch = blocks_per_step / 2
-        xu_peak = SM_COUNT * XU_PER_CLK_PER_SM * peaks.get("sm_max_mhz", NOMINAL_SM_MHZ) * 1e6
-        achieved = xu_ops_per_block(M, T_ITERS) * blocks_per_launch / mean_launch_s
-        achieved_lit = xu_ops_per_block_literal(M, T_ITERS) * blocks_per_launch / mean_launch_s
+        clk_hz = peaks.get("sm_max_mhz", NOMINAL_SM_MHZ) * 1e6
+        fma_peak = SM_COUNT * FMA_LANES_PER_CLK_PER_SM * clk_hz
+        xu_peak = SM_COUNT * XU_PER_CLK_PER_SM * clk_hz
+        achieved = fma_lane_ops_per_block(M, T_ITERS) * blocks_per_launch / mean_launch_s
+        t_sfu_one_exp = xu_ops_per_block_one_exp(M, T_ITERS) * blocks_per_launch / xu_peak
+        t_sfu_literal = xu_ops_per_block_literal(M, T_ITERS) * blocks_per_launch / xu_peak
         out = {
             "metric": "blocks_per_s", "value": value, "unit": "blocks/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
@@ -308,18 +322,22 @@ def run_cuda(args, rank, world, local_rank):
                     "d2h_bytes_per_step": sum(m.numel() * 4 for m in masks)},
             "gpu_launches": launches,
             "roofline": {
-                "bound": "alu", "pipe": "SFU (MUFU ex2/lg2/rcp)",
-                "achieved": achieved / 1e9, "peak": xu_peak / 1e9, "unit": "Gop/s",
-                "frac": achieved / xu_peak,
-                "frac_paper_literal_opcount": achieved_lit / xu_peak,
-                "peak_source": f"148 SMs x 16 SFU results/clk x sm_max_mhz ({peak_kind} clock)",
+                "bound": "alu", "pipe": "fp32 FMA pipe (add/mul/fma)",
+                "achieved": achieved / 1e12, "peak": fma_peak / 1e12, "unit": "Tlaneop/s",
+                "frac": achieved / fma_peak,
+                "peak_source": f"148 SMs x 128 fp32 lanes/clk x sm_max_mhz ({peak_kind} clock)",
                 "kernel": "tsenor_kernel<32,0>", "launch_ms": statistics.mean(launch_ms),
-                "traffic": None,
+                "traffic": NCU_DRAM_BYTES_PER_LAUNCH,
+                "algorithmic_bytes": bytes_per_step / 2 * (1 + 1 / 32),
                 "hbm_frac": (bytes_per_step / 2 * (1 + 1 / 32)) / mean_launch_s / 1e9 / peaks["hbm_gbs"],
+                # time the SFU alone would need for a log-domain iteration, over the measured time:
+                # how the kernel compares with the bounds the scope table was written against
+                "vs_sfu_bound_one_exp_per_element": t_sfu_one_exp / mean_launch_s,
+                "vs_sfu_bound_paper_listing": t_sfu_literal / mean_launch_s,
             },
         }
         if clocks and clocks.get("sm_mhz"):
-            out["roofline"]["frac_at_sampled_clock"] = achieved / (xu_peak * clocks["sm_mhz"] /
+            out["roofline"]["frac_at_sampled_clock"] = achieved / (fma_peak * clocks["sm_mhz"] /
                                                                    peaks.get("sm_max_mhz", NOMINAL_SM_MHZ))
         if not args.no_cpu_baseline and world == 1:
             rate, nblk, dt, cores = time_oracle(wls[0], args.cpu_blocks)

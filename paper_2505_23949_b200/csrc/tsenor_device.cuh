@@ -120,22 +120,31 @@ struct Comp {
 //     kap_j  = N / sum_i e_ij rho_i                (projection on C2)
 //     U_ij  <- U_ij rho_i kap_j ,  F_i += log2 rho_i ,  G_j += log2 kap_j
 // with the clip (C3) and the dual update implicit in the next e.  U is the
-// linear-domain iterate of Algorithm 1; it is only trusted for RESYNC
-// iterations at a time and then rebuilt as 2^(t0 + F + G) from the log-domain
-// potentials, which is what keeps large tau |w| safe in fp32: an entry that
-// overflowed stays clipped and one that flushed to zero stays negligible for
-// that long, because from iteration 1 on every rho*kap lies in
-// [N/M^3, N M^2] (row sums of e are in [1/M, M], column sums of e*rho in
-// [N/M, N M^2]).  Iteration 0 has no clip yet and is done entirely in the
-// log domain with the column maximum subtracted, because 2^t0 of a whole
-// column can underflow against a large entry elsewhere in its rows.
+// linear-domain iterate of Algorithm 1.  It is trusted only while the scalings
+// applied since it was last rebuilt stay small, and is then rebuilt as
+// 2^(t0 + F + G) from the log-domain potentials; that is what keeps large
+// tau |w| safe in fp32.  Every CHECK iterations the products of rho_i and of
+// kap_j since the last rebuild are tested against [2^-16, 2^17), and U is
+// rebuilt when one of them has left that range or after MAXRUN iterations.
+// From iteration 1 on every rho*kap lies in [N/M^3, N M^2], below 2^15 in
+// magnitude (row sums of e are in [1/M, M], column sums of e*rho in
+// [N/M, N M^2]), so between two rebuilds no entry moves by more than
+// 2^(34 + 15 CHECK) = 2^94 relative to its value at the last rebuild: an
+// entry that overflowed to +inf is still above the cap, and one that flushed
+// to zero (below 2^-126) is still below 2^-32, when the rebuild restores it
+// (in practice the scalings are within a few percent of 1 after the first
+// dozen iterations and the runs reach MAXRUN).  Iteration 0 has no clip yet and is done
+// entirely in the log domain with the column maximum subtracted, because
+// 2^t0 of a whole column can underflow against a large entry elsewhere in
+// its rows.
 //
 // On entry t holds t0 with its row maximum subtracted (exact no-op for the
 // method: the first row projection removes any row constant); on return t
 // holds the final t = x + q.  stash: 32 * MR * MC floats of shared memory
 // private to the warp (keeps t0 while the registers hold U).
 // ---------------------------------------------------------------------------
-constexpr int RESYNC = 6;   // (N M^2)^6 < 2^90: a flushed entry stays below 2^-36
+constexpr int CHECK = 4;     // iterations between range tests of the accumulated scalings
+constexpr int MAXRUN = 24;   // longest run of linear-domain iterations (multiple of CHECK)
 
 template <int M>
 __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>::MC], float* stash, int lane,
@@ -201,10 +210,20 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>:
     // Iterations 1 .. iters-1.  Element-wise work runs on pairs of columns with
     // the packed fp32x2 add / mul / fma of sm_100 (half the issue slots).
     float2 U[MR][MP];
-    int until_resync = 0;
+    int run = MAXRUN;                          // linear-domain iterations since the last rebuild
     for (int it = 1; it < iters; ++it) {
-        if (until_resync == 0) {
-            until_resync = RESYNC;
+        bool rebuild = (run >= MAXRUN);
+        if (!rebuild && (run % CHECK) == 0) {
+            // exponent field in [127-16, 127+16] <=> product in [2^-16, 2^17)
+            bool wide = false;
+#pragma unroll
+            for (int k = 0; k < RO; ++k) wide |= (((__float_as_uint(Pr[k]) >> 23) & 0xffu) - 111u) > 32u;
+#pragma unroll
+            for (int k = 0; k < CO; ++k) wide |= (((__float_as_uint(Pc[k]) >> 23) & 0xffu) - 111u) > 32u;
+            rebuild = __any_sync(FULL, wide);
+        }
+        if (rebuild) {
+            run = 0;
 #pragma unroll
             for (int k = 0; k < RO; ++k) { Fo[k].add(lg2_approx(Pr[k])); Pr[k] = 1.0f; F[k] = Fo[k].hi; }
 #pragma unroll
@@ -223,7 +242,7 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>:
                 U[a][b + 1] = make_float2(ex2_approx(x1.x), ex2_approx(x1.y));
             }
         }
-        --until_resync;
+        ++run;
         float2 e[MR][MP];
         float rp[MR], rho[MR], cp[MC], kap[MC];
 #pragma unroll
