@@ -32,7 +32,7 @@ XU_PER_CLK_PER_SM = 16          # special-function results per clock per SM
 NOMINAL_SM_MHZ = 1965.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one tsenor_kernel<32,0> launch on the
 # 14336x4096 matrix, from the ncu capture summarised under profiles/ (None until captured)
-NCU_DRAM_BYTES_PER_LAUNCH = None
+NCU_DRAM_BYTES_PER_LAUNCH = 243.78e6   # 234.99 MB read + 8.79 MB written
 
 
 def fma_lane_ops_per_block(M, T):
@@ -115,6 +115,27 @@ class ClockSampler:
         return {"sm_mhz": statistics.median(self.samples), "sm_min_mhz": min(self.samples),
                 "sm_max_mhz": self.smax, "reasons": reasons, "samples": len(self.samples),
                 "power_w_max": max(self.power) if self.power else None}
+
+
+def rank_workload_index(rank):
+    """Weak scaling: every rank solves its own copy of the workload; the seed index is the rank."""
+    return int(rank)
+
+
+def max_over_ranks(value, world, device=None):
+    """Largest per-rank value (elapsed time): one scalar all-reduce, outside any timed region."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_rate(units_per_rank_per_step, steps, world, elapsed_ms):
+    """Whole-job throughput: units all ranks processed over the slowest rank's time."""
+    return world * units_per_rank_per_step * steps / (elapsed_ms / 1e3)
 
 
 def make_workload(index):
@@ -200,7 +221,7 @@ def run_cuda(args, rank, world, local_rank):
         dist.init_process_group("nccl", device_id=dev)
     ts.lib()  # fail loudly if the CUDA library is missing
 
-    wls = make_workload(rank)
+    wls = make_workload(rank_workload_index(rank))
     host = [torch.from_numpy(w.scores).pin_memory() for w in wls]
     taus = [synth.default_tau(float(w.scores.max())) for w in wls]
     dev_scores = [h.to(dev, non_blocking=True) for h in host]
@@ -268,10 +289,7 @@ def run_cuda(args, rank, world, local_rank):
     clocks = sampler.stop() if sampler else None
     total_ms = ev[0].elapsed_time(ev[-1])
     launch_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(2 * args.steps)]
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world, dev)
     flags = int(status.item())
     bad = sum(int(ts.check(m, *w.scores.shape, w.N, w.M).item()) for m, w in zip(masks, wls))
 
@@ -292,15 +310,12 @@ def run_cuda(args, rank, world, local_rank):
     e1.record(cur)
     barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, world, dev)
 
     if rank == 0:
         peaks, peak_kind = measured_peaks()
         sec = total_ms / 1e3
-        value = world * blocks_per_step * args.steps / sec
+        value = aggregate_rate(blocks_per_step, args.steps, world, total_ms)
         mean_launch_s = statistics.mean(launch_ms) / 1e3
         blocks_per_launch = blocks_per_step / 2
         clk_hz = peaks.get("sm_max_mhz", NOMINAL_SM_MHZ) * 1e6
@@ -317,7 +332,7 @@ def run_cuda(args, rank, world, local_rank):
             "gb_scores_per_s": world * bytes_per_step * args.steps / sec / 1e9,
             "infeasible_blocks": bad, "dev_status": flags,
             "clocks": clocks,
-            "e2e": {"value": world * blocks_per_step * args.steps / (e2e_ms / 1e3), "unit": "blocks/s",
+            "e2e": {"value": aggregate_rate(blocks_per_step, args.steps, world, e2e_ms), "unit": "blocks/s",
                     "h2d_bytes_per_step": bytes_per_step,
                     "d2h_bytes_per_step": sum(m.numel() * 4 for m in masks)},
             "gpu_launches": launches,
