@@ -143,6 +143,9 @@ struct Comp {
 // holds the final t = x + q.  stash: 32 * MR * MC floats of shared memory
 // private to the warp (keeps t0 while the registers hold U).
 // ---------------------------------------------------------------------------
+// Whether the row scalings are folded into the clip threshold instead of the tile
+// (one multiply per element less, three shuffles more): pays off except at M = 32.
+template <int M> struct LazyRow { static constexpr bool value = (M != 32); };
 constexpr int CHECK = 4;     // iterations between range tests of the accumulated scalings
 constexpr int MAXRUN = 24;   // longest run of linear-domain iterations (multiple of CHECK)
 
@@ -210,6 +213,8 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>:
     // Iterations 1 .. iters-1.  Element-wise work runs on pairs of columns with
     // the packed fp32x2 add / mul / fma of sm_100 (half the issue slots).
     float2 U[MR][MP];
+    float iR[MR];
+    const float invN = 1.0f / Nf;
     int run = MAXRUN;                          // linear-domain iterations since the last rebuild
     for (int it = 1; it < iters; ++it) {
         bool rebuild = (run >= MAXRUN);
@@ -243,6 +248,56 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>:
             }
         }
         ++run;
+      if (LazyRow<M>::value) {
+        // Row scalings stay out of the tile: it holds V = U / R_i (R_i = product of the
+        // rho_i since the rebuild), e = R_i min(V, 1/R_i); the new R_i is N / sum_j min(..).
+        if (rebuild) {
+#pragma unroll
+            for (int a = 0; a < MR; ++a) iR[a] = 1.0f;
+        }
+        float2 m[MR][MP];
+        float rp[MR], Rn[MR], iRn[MR], cp[MC], kap[MC];
+#pragma unroll
+        for (int a = 0; a < MR; ++a) {
+            float2 s2;
+#pragma unroll
+            for (int b = 0; b < MP; ++b) {
+                m[a][b] = make_float2(fminf(U[a][b].x, iR[a]), fminf(U[a][b].y, iR[a]));
+                s2 = (b == 0) ? m[a][b] : __fadd2_rn(s2, m[a][b]);
+            }
+            rp[a] = s2.x + s2.y;
+        }
+        reduce_scatter<MR, PC>(rp, 1, OpAdd());
+#pragma unroll
+        for (int k = 0; k < RO; ++k) {
+            Pr[k] = Nf * rcp_approx(rp[k]);
+            Rn[k] = Pr[k];
+            iRn[k] = rp[k] * invN;
+        }
+        all_gather<MR, PC>(Rn, 1);
+        all_gather<MR, PC>(iRn, 1);
+#pragma unroll
+        for (int b = 0; b < MP; ++b) {
+            float2 c2 = __fmul2_rn(m[0][b], make_float2(Rn[0], Rn[0]));
+#pragma unroll
+            for (int a = 1; a < MR; ++a) c2 = __ffma2_rn(m[a][b], make_float2(Rn[a], Rn[a]), c2);
+            cp[2 * b] = c2.x;
+            cp[2 * b + 1] = c2.y;
+        }
+        reduce_scatter<MC, PR>(cp, PC, OpAdd());
+#pragma unroll
+        for (int k = 0; k < CO; ++k) {
+            kap[k] = Nf * rcp_approx(cp[k]);
+            Pc[k] *= kap[k];
+        }
+        all_gather<MC, PR>(kap, PC);
+#pragma unroll
+        for (int a = 0; a < MR; ++a) {
+            iR[a] = iRn[a];
+#pragma unroll
+            for (int b = 0; b < MP; ++b) U[a][b] = __fmul2_rn(U[a][b], make_float2(kap[2 * b], kap[2 * b + 1]));
+        }
+      } else {
         float2 e[MR][MP];
         float rp[MR], rho[MR], cp[MC], kap[MC];
 #pragma unroll
@@ -284,6 +339,7 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>:
             for (int b = 0; b < MP; ++b)
                 U[a][b] = __fmul2_rn(__fmul2_rn(U[a][b], ra), make_float2(kap[2 * b], kap[2 * b + 1]));
         }
+      }
     }
     // final potentials and t = t0 + F + G
 #pragma unroll
