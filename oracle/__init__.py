@@ -59,6 +59,12 @@ def lib():
         L.oracle_block_objectives.restype = i32
         L.oracle_max_abs.argtypes = [_f32p, i64, i64, i64]
         L.oracle_max_abs.restype = f32
+        L.oracle_scores.argtypes = [i32, _f32p, i64, vp, i64, f32, vp, i64, i64, _f32p, i64]
+        L.oracle_scores.restype = i32
+        L.oracle_keep_better.argtypes = [_f32p, i64, i64, i64, _u32p, _u32p, _f64p]
+        L.oracle_keep_better.restype = i32
+        L.oracle_simple_round.argtypes = [_f32p, i64, i64, i64, i32, i32, _u32p]
+        L.oracle_simple_round.restype = i32
         L.oracle_num_threads.argtypes = []
         L.oracle_num_threads.restype = i32
         _lib = L
@@ -234,6 +240,46 @@ def block_objectives(scores, bits, M):
 def max_abs(scores):
     s = _f32(scores)
     return float(lib().oracle_max_abs(s, s.shape[0], s.shape[1], s.shape[1]))
+
+
+SCORES_ABS, SCORES_ADMM, SCORES_COLDIV, SCORES_COLMUL = 0, 1, 2, 3
+
+
+def scores(kind, w, v=None, scalar=0.0, colvec=None):
+    """Score matrix of a pruning framework (Section 4): |W|, the ADMM D-update score
+    (W + V*scalar)^2 with scalar = 1/rho, the SparseGPT group score |W_ij / d_j|, or the
+    Wanda score |W_ij| a_j.  fp32 in, fp32 out, one rounding per operation."""
+    w = _f32(w)
+    rows, cols = w.shape
+    out = np.empty((rows, cols), np.float32)
+    vv = None if v is None else _f32(v)
+    cv = None if colvec is None else _f32(colvec)
+    rc = lib().oracle_scores(int(kind), w, cols,
+                             None if vv is None else vv.ctypes.data_as(C.c_void_p), cols,
+                             float(scalar), None if cv is None else cv.ctypes.data_as(C.c_void_p),
+                             rows, cols, out, cols)
+    _check(rc, "scores")
+    return out
+
+
+def keep_better(score_matrix, prev_mask, new_mask):
+    """Safeguard of the ADMM integration (Appendix A.1.3): the new mask unless it retains
+    less score than the previous one.  Returns ``(kept_mask, obj_new, obj_prev)``."""
+    s = _f32(score_matrix)
+    prev = np.ascontiguousarray(prev_mask, dtype=np.uint32)
+    kept = np.array(new_mask, dtype=np.uint32, order="C", copy=True)
+    obj2 = np.zeros(2, np.float64)
+    _check(lib().oracle_keep_better(s, s.shape[1], s.shape[0], s.shape[1], prev, kept, obj2), "keep_better")
+    return kept, float(obj2[0]), float(obj2[1])
+
+
+def simple_round(plan_key, N, M):
+    """"Simple" rounding of the ablation study: row-wise then column-wise N:M rounding."""
+    k = _f32(plan_key)
+    rows, cols = k.shape
+    bits = np.zeros((rows, mask_words_per_row(cols)), np.uint32)
+    _check(lib().oracle_simple_round(k, cols, rows, cols, int(N), int(M), bits), "simple_round")
+    return bits
 
 
 def num_threads():

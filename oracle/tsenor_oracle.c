@@ -612,3 +612,111 @@ int oracle_num_threads(void)
 #endif
     return n;
 }
+
+/* ------------------------------------------------------------------ */
+/* Score matrices of the pruning frameworks (Section 4) and the mask    */
+/* safeguard of the ADMM integration (Appendix A.1.3)                   */
+/* ------------------------------------------------------------------ */
+
+/* kinds: 0 |W|; 1 ADMM D-update (W + V/rho)^2 (Proposition 1); 2 SparseGPT
+ * group score |W_ij / d_j| with d_j = [H^-1]_jj (the printed -W/[H^-1]_jj,
+ * magnitude taken); 3 Wanda |W_ij| a_j with a_j the input-feature norm.
+ * Every product, sum and quotient is one fp32 operation (no fused
+ * multiply-add), so that an fp32 implementation yields the same bits.
+ * W is fp32 here; for kind 3 the caller passes bf16 weights widened to fp32
+ * (exact). */
+int oracle_scores(int kind, const float *w, int64_t ld, const float *v,
+                  int64_t ld_v, float scalar, const float *colvec, int64_t rows,
+                  int64_t cols, float *out, int64_t ld_out)
+{
+    if (!w || !out || rows < 0 || cols < 0) return ORACLE_ERR_ARG;
+    if (kind == 1 && !v) return ORACLE_ERR_ARG;
+    if ((kind == 2 || kind == 3) && !colvec) return ORACLE_ERR_ARG;
+    if (kind < 0 || kind > 3) return ORACLE_ERR_ARG;
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t c = 0; c < cols; ++c) {
+            volatile float x = w[(size_t)r * ld + c], y;
+            if (kind == 0) {
+                y = fabsf(x);
+            } else if (kind == 1) {
+                volatile float t = v[(size_t)r * ld_v + c] * scalar; /* V / rho */
+                volatile float s = x + t;
+                y = s * s;
+            } else if (kind == 2) {
+                volatile float q = x / colvec[c];
+                y = fabsf(q);
+            } else {
+                volatile float a = fabsf(x);
+                y = a * colvec[c];
+            }
+            out[(size_t)r * ld_out + c] = y;
+        }
+    return ORACLE_OK;
+}
+
+/* Safeguard of the ADMM integration: keep the previous mask whenever the new
+ * one retains less score.  mask_inout holds the new mask on entry and the
+ * kept one on return; obj2 receives {objective(new), objective(previous)}. */
+int oracle_keep_better(const float *scores, int64_t ld, int64_t rows,
+                       int64_t cols, const uint32_t *prev_mask,
+                       uint32_t *mask_inout, double *obj2)
+{
+    if (!scores || !prev_mask || !mask_inout) return ORACLE_ERR_ARG;
+    double on = oracle_objective(scores, ld, mask_inout, rows, cols);
+    double op = oracle_objective(scores, ld, prev_mask, rows, cols);
+    if (on < op)
+        memcpy(mask_inout, prev_mask,
+               sizeof(uint32_t) * (size_t)(rows * ((cols + 31) / 32)));
+    if (obj2) {
+        obj2[0] = on;
+        obj2[1] = op;
+    }
+    return ORACLE_OK;
+}
+
+/* "Simple" rounding of the ablation study (Appendix B.2): row-wise N:M
+ * rounding of the plan (keep the N largest keys of every row of the block),
+ * then column-wise N:M rounding of what is left (keep the N largest of every
+ * column among the survivors).  Ties by ascending index.  The result has at
+ * most N per line and may be under-filled. */
+int oracle_simple_round(const float *plan_key, int64_t ld_plan, int64_t rows,
+                        int64_t cols, int N, int M, uint32_t *mask_bits)
+{
+    if (!plan_key || !mask_bits || !check_shape(rows, cols, N, M) || N < 1 ||
+        N >= M)
+        return ORACLE_ERR_ARG;
+    int64_t nbr = rows / M, nbc = cols / M, wpr = (cols + 31) / 32;
+    memset(mask_bits, 0, sizeof(uint32_t) * (size_t)(rows * wpr));
+    uint8_t *S = (uint8_t *)malloc((size_t)M * M);
+    sort_item *it = (sort_item *)malloc(sizeof(sort_item) * (size_t)M);
+    for (int64_t br = 0; br < nbr; ++br)
+        for (int64_t bc = 0; bc < nbc; ++bc) {
+            int64_t r0 = br * M, c0 = bc * M;
+            memset(S, 0, (size_t)M * M);
+            for (int i = 0; i < M; ++i) { /* row-wise N:M */
+                for (int j = 0; j < M; ++j) {
+                    double k = plan_key[(size_t)(r0 + i) * ld_plan + c0 + j];
+                    it[j].key = (k != k) ? -INFINITY : k;
+                    it[j].idx = j;
+                }
+                qsort(it, (size_t)M, sizeof(sort_item), cmp_desc_key_then_index);
+                for (int t = 0; t < N; ++t) S[i * M + it[t].idx] = 1;
+            }
+            for (int j = 0; j < M; ++j) { /* column-wise N:M on the survivors */
+                int n = 0;
+                for (int i = 0; i < M; ++i)
+                    if (S[i * M + j]) {
+                        double k = plan_key[(size_t)(r0 + i) * ld_plan + c0 + j];
+                        it[n].key = (k != k) ? -INFINITY : k;
+                        it[n].idx = i;
+                        n++;
+                    }
+                qsort(it, (size_t)n, sizeof(sort_item), cmp_desc_key_then_index);
+                for (int t = N; t < n; ++t) S[it[t].idx * M + j] = 0;
+            }
+            store_block_bits(S, M, r0, c0, wpr, mask_bits);
+        }
+    free(S);
+    free(it);
+    return ORACLE_OK;
+}

@@ -412,3 +412,74 @@ def test_mask_bit_layout_and_helpers():
     assert oracle.max_abs(-W) == 7.0
     with pytest.raises(ValueError):
         oracle.solve(np.zeros((6, 8), np.float32), 2, 4, 1.0, 1)
+
+
+# ------------------------------------- framework scores, safeguard, simple rounding
+
+def test_framework_score_formulas():
+    rng = np.random.default_rng(31)
+    W = rng.standard_normal((24, 40)).astype(np.float32)
+    V = rng.standard_normal((24, 40)).astype(np.float32)
+    rho = 3.0
+    s = oracle.scores(oracle.SCORES_ADMM, W, V, 1.0 / rho)
+    ref = (W.astype(np.float64) + V.astype(np.float64) / rho) ** 2
+    assert np.allclose(s, ref, rtol=1e-6, atol=1e-9)
+    # D-update of Proposition 1: with D = (W + V/rho) .* S the distance to W + V/rho is the
+    # score mass left outside the mask, so maximising the retained score minimises it
+    S = (rng.random((24, 40)) < 0.5)
+    Z = W.astype(np.float64) + V.astype(np.float64) / rho
+    assert np.isclose(((Z * S - Z) ** 2).sum(), (ref * (~S)).sum(), rtol=1e-12)
+    X = rng.standard_normal((64, 40))
+    a = np.linalg.norm(X, axis=0).astype(np.float32)          # input-feature norms (Wanda)
+    assert np.allclose(oracle.scores(oracle.SCORES_COLMUL, W, colvec=a), np.abs(W) * a, rtol=1e-7)
+    d = (np.abs(rng.standard_normal(40)) + 0.1).astype(np.float32)
+    assert np.allclose(oracle.scores(oracle.SCORES_COLDIV, W, colvec=d), np.abs(-W / d), rtol=1e-7)
+    assert np.array_equal(oracle.scores(oracle.SCORES_ABS, W), np.abs(W))
+
+
+def test_keep_better_never_lowers_the_objective():
+    rng = np.random.default_rng(32)
+    M, N = 8, 4
+    W = rng.standard_normal((32, 64)).astype(np.float32)
+    prev = None
+    for t in range(6):                                    # a drifting score matrix, as in ADMM
+        V = (0.3 * t) * rng.standard_normal(W.shape).astype(np.float32)
+        sc = oracle.scores(oracle.SCORES_ADMM, W, V, 0.5)
+        new = oracle.solve(sc, N, M, 200.0 / sc.max(), 60)
+        if prev is None:
+            prev = new
+            continue
+        if t == 3:                                        # force the other branch once
+            new = oracle.round_plan(-sc, sc, N, M)        # a deliberately poor mask
+        kept, o_new, o_prev = oracle.keep_better(sc, prev, new)
+        assert o_new == oracle.objective(sc, new) and o_prev == oracle.objective(sc, prev)
+        assert oracle.objective(sc, kept) == max(o_new, o_prev)
+        assert np.array_equal(kept, new if o_new >= o_prev else prev)
+        if t == 3:
+            assert o_new < o_prev
+        prev = kept
+
+
+def test_simple_rounding_properties_and_ablation_order():
+    rng = np.random.default_rng(33)
+    M, N, nb = 8, 4, 8
+    W = np.abs(rng.standard_normal((M * nb, M * nb)) * 0.02).astype(np.float32)
+    tau = 200.0 / W.max()
+    x = oracle.dykstra(W, N, M, tau, 300, plan_is_log=True).astype(np.float32)
+    simple = oracle.unpack_mask(oracle.simple_round(x, N, M), M * nb)
+    for b in range(nb * nb):
+        r0, c0 = (b // nb) * M, (b % nb) * M
+        S = simple[r0:r0 + M, c0:c0 + M]
+        k = x[r0:r0 + M, c0:c0 + M]
+        assert S.sum(0).max() <= N and S.sum(1).max() <= N
+        for i in range(M):                                # survivors come from the row's top N
+            top = sorted(range(M), key=lambda j: (-k[i, j], j))[:N]
+            assert set(np.flatnonzero(S[i])) <= set(top)
+    # a plan that already is a feasible mask is returned unchanged
+    feas = oracle.unpack_mask(oracle.solve(W, N, M, tau, 300), M * nb).astype(np.float32)
+    assert np.array_equal(oracle.unpack_mask(oracle.simple_round(feas, N, M), M * nb), feas.astype(np.uint8))
+    # ablation order of Appendix B.2 on the same plan: simple <= greedy only <= greedy + local search
+    o_simple = (simple * W.astype(np.float64)).sum()
+    o_greedy = oracle.objective(W, oracle.round_plan(x, W, N, M, ls_steps=0))
+    o_full = oracle.objective(W, oracle.round_plan(x, W, N, M))
+    assert o_simple < o_greedy <= o_full
