@@ -423,7 +423,7 @@ def test_framework_score_formulas():
     rho = 3.0
     s = oracle.scores(oracle.SCORES_ADMM, W, V, 1.0 / rho)
     ref = (W.astype(np.float64) + V.astype(np.float64) / rho) ** 2
-    assert np.allclose(s, ref, rtol=1e-6, atol=1e-9)
+    assert np.allclose(s, ref, rtol=1e-5, atol=1e-6)          # three fp32 roundings, cancellation in the sum
     # D-update of Proposition 1: with D = (W + V/rho) .* S the distance to W + V/rho is the
     # score mass left outside the mask, so maximising the retained score minimises it
     S = (rng.random((24, 40)) < 0.5)
