@@ -109,7 +109,9 @@ int tsenor_round(const float *plan_key, int64_t ld_plan, const float *scores,
 
 /*
  * Objective of Eq. 1: *dev_sum_out (one double on the device, overwritten) =
- * sum of |scores[r][c]| over the set bits of the mask, accumulated in fp64.
+ * sum of |scores[r][c]| over the set bits of the mask, accumulated in fp64
+ * with atomic adds.  cols must be a multiple of 4 (it is for every mask the
+ * solver produces).
  */
 int tsenor_objective(const float *scores, int64_t ld, const uint32_t *mask_bits,
                      int64_t rows, int64_t cols, double *dev_sum_out,
@@ -125,11 +127,79 @@ int tsenor_check(const uint32_t *mask_bits, int64_t rows, int64_t cols, int N,
 
 /*
  * *dev_max_out (one float on the device, overwritten) = max |scores[r][c]|
- * (NaN entries are ignored).  Helper for the paper's parameter choice, which
+ * (NaN entries are ignored; cols a multiple of 4).  Helper for the paper's parameter choice, which
  * ties tau to the largest magnitude of the matrix (Appendix B.1).
  */
 int tsenor_max_abs(const float *scores, int64_t rows, int64_t cols, int64_t ld,
                    float *dev_max_out, tsenor_stream_t stream);
+
+/* ------------------------------------------------------------------------
+ * Score matrices of the pruning frameworks the solver plugs into (Section 4),
+ * computed in the block loader so that no score matrix is materialised.
+ * Every product, sum and quotient below is one fp32 operation (no fused
+ * multiply-add).  The descriptor itself is a HOST struct; the pointers in it
+ * are device pointers.
+ * ---------------------------------------------------------------------- */
+enum {
+    TSENOR_SCORES_ABS = 0,    /* |W_ij|                       magnitude pruning        */
+    TSENOR_SCORES_ADMM = 1,   /* (W_ij + V_ij * scalar)^2     D-update of the ADMM
+                                 integration, scalar = 1/rho (Proposition 1)           */
+    TSENOR_SCORES_COLDIV = 2, /* |W_ij / colvec_j|            SparseGPT group score,
+                                 colvec_j = [H^-1]_jj (the printed -W/[H^-1]_jj,
+                                 magnitude taken)                                      */
+    TSENOR_SCORES_COLMUL = 3  /* |W_ij| * colvec_j            Wanda score, colvec_j =
+                                 norm of input feature j; W may be bf16               */
+};
+
+typedef struct tsenor_scores {
+    int kind;            /* one of TSENOR_SCORES_*                                     */
+    int w_is_bf16;       /* non-zero: w points to bf16 (only with TSENOR_SCORES_COLMUL) */
+    const void *w;       /* rows x cols weights, row-major, leading dimension ld       */
+    int64_t ld;
+    const float *v;      /* TSENOR_SCORES_ADMM: dual variable V, rows x cols fp32      */
+    int64_t ld_v;
+    float scalar;        /* TSENOR_SCORES_ADMM: 1/rho                                  */
+    const float *colvec; /* COLDIV / COLMUL: cols floats                               */
+} tsenor_scores_t;
+
+/* tsenor_solve on the score matrix described by *s (same arguments otherwise). */
+int tsenor_solve_scores(const tsenor_scores_t *s, int64_t rows, int64_t cols,
+                        int N, int M, float tau, int iters, int ls_steps,
+                        uint32_t *mask_bits_out, int32_t *dev_status,
+                        tsenor_stream_t stream);
+
+/* *dev_max_out = largest score of the described matrix (for the choice of tau). */
+int tsenor_scores_max(const tsenor_scores_t *s, int64_t rows, int64_t cols,
+                      float *dev_max_out, tsenor_stream_t stream);
+
+/* Writes the described scores as fp32 (rows x cols, leading dimension ld_out):
+ * for tests, and to feed tsenor_round / tsenor_dykstra. */
+int tsenor_scores_materialize(const tsenor_scores_t *s, int64_t rows,
+                              int64_t cols, float *scores_out, int64_t ld_out,
+                              tsenor_stream_t stream);
+
+/*
+ * Safeguard of the ADMM integration (Appendix A.1.3): keep the previous mask
+ * whenever the new one retains less score under the current score matrix.
+ * mask_inout holds the new mask on entry and the kept one on return;
+ * dev_obj2_out (two doubles on the device, overwritten) receives
+ * {objective(new), objective(previous)}, accumulated in fp64 with atomic adds
+ * (summation order, hence the last bits, may vary between runs).
+ */
+int tsenor_keep_better(const tsenor_scores_t *s, int64_t rows, int64_t cols,
+                       const uint32_t *prev_mask, uint32_t *mask_inout,
+                       double *dev_obj2_out, tsenor_stream_t stream);
+
+/*
+ * "Simple" rounding of the ablation study (Appendix B.2): row-wise N:M
+ * rounding of the plan inside every block (keep the N largest keys of each
+ * row), then column-wise N:M rounding of the survivors.  Same key order and
+ * mask layout as tsenor_round; the result has at most N per line.
+ * Requires 0 < N < M.
+ */
+int tsenor_simple_round(const float *plan_key, int64_t ld_plan, int64_t rows,
+                        int64_t cols, int N, int M, uint32_t *mask_bits_out,
+                        tsenor_stream_t stream);
 
 /* ceil(cols / 32): uint32 words per mask row (host arithmetic only). */
 int64_t tsenor_mask_words_per_row(int64_t cols);

@@ -20,8 +20,17 @@ DEV_NONFINITE_SCORE, DEV_UNDERFILLED, DEV_INTERNAL = 1, 2, 4
 EXPORTS = (
     "tsenor_solve", "tsenor_dykstra", "tsenor_round", "tsenor_objective", "tsenor_check",
     "tsenor_max_abs", "tsenor_mask_words_per_row", "tsenor_strerror", "tsenor_last_cuda_error",
-    "tsenor_launch_count",
+    "tsenor_launch_count", "tsenor_solve_scores", "tsenor_scores_max", "tsenor_scores_materialize",
+    "tsenor_keep_better", "tsenor_simple_round",
 )
+
+SCORES_ABS, SCORES_ADMM, SCORES_COLDIV, SCORES_COLMUL = 0, 1, 2, 3
+
+
+class ScoresDesc(C.Structure):
+    """ctypes image of ``tsenor_scores_t`` (a host struct holding device pointers)."""
+    _fields_ = [("kind", C.c_int), ("w_is_bf16", C.c_int), ("w", C.c_void_p), ("ld", C.c_int64),
+                ("v", C.c_void_p), ("ld_v", C.c_int64), ("scalar", C.c_float), ("colvec", C.c_void_p)]
 
 _lib = None
 
@@ -53,6 +62,15 @@ def lib():
         L.tsenor_max_abs.argtypes = [vp, i64, i64, i64, vp, vp]
         for name in ("tsenor_solve", "tsenor_dykstra", "tsenor_round", "tsenor_objective",
                      "tsenor_check", "tsenor_max_abs", "tsenor_last_cuda_error"):
+            getattr(L, name).restype = i32
+        sp = C.POINTER(ScoresDesc)
+        L.tsenor_solve_scores.argtypes = [sp, i64, i64, i32, i32, f32, i32, i32, vp, vp, vp]
+        L.tsenor_scores_max.argtypes = [sp, i64, i64, vp, vp]
+        L.tsenor_scores_materialize.argtypes = [sp, i64, i64, vp, i64, vp]
+        L.tsenor_keep_better.argtypes = [sp, i64, i64, vp, vp, vp, vp]
+        L.tsenor_simple_round.argtypes = [vp, i64, i64, i64, i32, i32, vp, vp]
+        for name in ("tsenor_solve_scores", "tsenor_scores_max", "tsenor_scores_materialize",
+                     "tsenor_keep_better", "tsenor_simple_round"):
             getattr(L, name).restype = i32
         L.tsenor_mask_words_per_row.argtypes = [i64]
         L.tsenor_mask_words_per_row.restype = i64
@@ -168,3 +186,93 @@ def max_abs(scores, out=None, stream=None):
     if rc:
         raise TsenorError(rc, "tsenor_max_abs")
     return out
+
+
+class Scores:
+    """A described score matrix (``tsenor_scores_t``): keeps the tensors alive and builds
+    the descriptor.  kind: SCORES_ABS |W|, SCORES_ADMM (W + V*scalar)^2, SCORES_COLDIV
+    |W / colvec_j|, SCORES_COLMUL |W| * colvec_j (W may be bfloat16)."""
+
+    def __init__(self, kind, w, v=None, scalar=0.0, colvec=None):
+        if not (isinstance(w, torch.Tensor) and w.is_cuda and w.dim() == 2 and w.stride(1) == 1):
+            raise TypeError("w must be a 2-D row-major CUDA tensor")
+        if w.dtype not in (torch.float32, torch.bfloat16):
+            raise TypeError("w must be float32 or bfloat16")
+        self.kind, self.w, self.v, self.colvec = int(kind), w, v, colvec
+        self.rows, self.cols = w.shape
+        d = ScoresDesc()
+        d.kind = self.kind
+        d.w_is_bf16 = int(w.dtype == torch.bfloat16)
+        d.w = w.data_ptr()
+        d.ld = w.stride(0) if self.rows > 1 else max(w.stride(0), self.cols)
+        if v is not None:
+            _, r2, c2, ldv = _mat(v, "v")
+            if (r2, c2) != (self.rows, self.cols):
+                raise ValueError("v and w differ in shape")
+            d.v, d.ld_v = v.data_ptr(), ldv
+        d.scalar = float(scalar)
+        if colvec is not None:
+            if not (colvec.is_cuda and colvec.dtype == torch.float32 and colvec.is_contiguous()
+                    and colvec.numel() == self.cols):
+                raise TypeError("colvec must be a contiguous float32 CUDA vector of length cols")
+            d.colvec = colvec.data_ptr()
+        self.desc = d
+
+    @property
+    def device(self):
+        return self.w.device
+
+
+def solve_scores(src, N, M, tau, iters=300, ls_steps=-1, mask_out=None, status=None, stream=None):
+    """tsenor_solve_scores: the whole method on a described score matrix."""
+    if mask_out is None:
+        mask_out = new_mask(src.rows, src.cols, src.device)
+    rc = lib().tsenor_solve_scores(C.byref(src.desc), src.rows, src.cols, int(N), int(M), float(tau), int(iters),
+                                   int(ls_steps), _ptr(mask_out), _ptr(status), _stream(stream))
+    if rc:
+        raise TsenorError(rc, "tsenor_solve_scores")
+    return mask_out
+
+
+def scores_max(src, out=None, stream=None):
+    """tsenor_scores_max: 1-element float32 device tensor with the largest score."""
+    if out is None:
+        out = torch.empty(1, dtype=torch.float32, device=src.device)
+    rc = lib().tsenor_scores_max(C.byref(src.desc), src.rows, src.cols, _ptr(out), _stream(stream))
+    if rc:
+        raise TsenorError(rc, "tsenor_scores_max")
+    return out
+
+
+def scores_materialize(src, out=None, stream=None):
+    """tsenor_scores_materialize: the described scores as a float32 matrix."""
+    if out is None:
+        out = torch.empty((src.rows, src.cols), dtype=torch.float32, device=src.device)
+    p, _, _, ld = _mat(out, "out")
+    rc = lib().tsenor_scores_materialize(C.byref(src.desc), src.rows, src.cols, p, ld, _stream(stream))
+    if rc:
+        raise TsenorError(rc, "tsenor_scores_materialize")
+    return out
+
+
+def keep_better(src, prev_mask, mask_inout, obj2_out=None, stream=None):
+    """tsenor_keep_better: keeps ``prev_mask`` in ``mask_inout`` if it retains more score.
+    Returns the 2-element float64 device tensor {objective(new), objective(previous)}."""
+    if obj2_out is None:
+        obj2_out = torch.empty(2, dtype=torch.float64, device=src.device)
+    rc = lib().tsenor_keep_better(C.byref(src.desc), src.rows, src.cols, _ptr(prev_mask), _ptr(mask_inout),
+                                  _ptr(obj2_out), _stream(stream))
+    if rc:
+        raise TsenorError(rc, "tsenor_keep_better")
+    return obj2_out
+
+
+def simple_round(plan_key, N, M, mask_out=None, stream=None):
+    """tsenor_simple_round: row-wise then column-wise N:M rounding of the plan."""
+    pk, rows, cols, ldk = _mat(plan_key, "plan_key")
+    if mask_out is None:
+        mask_out = new_mask(rows, cols, plan_key.device)
+    rc = lib().tsenor_simple_round(pk, ldk, rows, cols, int(N), int(M), _ptr(mask_out), _stream(stream))
+    if rc:
+        raise TsenorError(rc, "tsenor_simple_round")
+    return mask_out

@@ -34,6 +34,43 @@ inline bool aligned16(const void* p, int64_t ld) {
     return (reinterpret_cast<uintptr_t>(p) % 16 == 0) && (ld % 4 == 0);
 }
 
+tsenor::ScoreSrc abs_source(const float* scores, int64_t ld) {
+    tsenor::ScoreSrc S{};
+    S.kind = tsenor::SC_ABS;
+    S.w = scores; S.ld = ld;
+    S.vec_w = aligned16(scores, ld);
+    return S;
+}
+
+// Validates a caller's descriptor and turns it into the device-side form.
+int make_source(const tsenor_scores_t* d, int64_t cols, tsenor::ScoreSrc* out) {
+    if (!d) return TSENOR_ERR_NULL;
+    if (d->kind < TSENOR_SCORES_ABS || d->kind > TSENOR_SCORES_COLMUL) return TSENOR_ERR_ARG;
+    if (d->w_is_bf16 && d->kind != TSENOR_SCORES_COLMUL) return TSENOR_ERR_ARG;
+    if (d->ld < cols) return TSENOR_ERR_SHAPE;
+    if (!d->w) return TSENOR_ERR_NULL;
+    tsenor::ScoreSrc S{};
+    S.kind = d->kind;
+    S.w_is_bf16 = d->w_is_bf16 ? 1 : 0;
+    S.w = d->w; S.ld = d->ld;
+    S.vec_w = d->w_is_bf16 ? ((reinterpret_cast<uintptr_t>(d->w) % 8 == 0) && (d->ld % 4 == 0))
+                           : aligned16(d->w, d->ld);
+    if (d->kind == TSENOR_SCORES_ADMM) {
+        if (!d->v) return TSENOR_ERR_NULL;
+        if (d->ld_v < cols) return TSENOR_ERR_SHAPE;
+        if (!std::isfinite(d->scalar)) return TSENOR_ERR_ARG;
+        S.v = d->v; S.ld_v = d->ld_v; S.scalar = d->scalar;
+        S.vec_v = aligned16(d->v, d->ld_v);
+    }
+    if (d->kind == TSENOR_SCORES_COLDIV || d->kind == TSENOR_SCORES_COLMUL) {
+        if (!d->colvec) return TSENOR_ERR_NULL;
+        S.colvec = d->colvec;
+        S.vec_c = (reinterpret_cast<uintptr_t>(d->colvec) % 16 == 0);
+    }
+    *out = S;
+    return TSENOR_OK;
+}
+
 template <int M, int MODE>
 int launch(const tsenor::Params& P, cudaStream_t st) {
     using G = tsenor::Geom<M>;
@@ -90,30 +127,133 @@ __global__ void fill_mask_kernel(uint32_t* bits, int64_t rows, int64_t wpr, int6
     }
 }
 
-__global__ void objective_kernel(const float* __restrict__ scores, int64_t ld, const uint32_t* __restrict__ bits,
-                                 int64_t rows, int64_t cols, int64_t wpr, double* out) {
-    double acc = 0.0;
-    const int64_t nwords = rows * wpr;
-    for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < nwords;
+// Retained score of up to two masks under one score source (quads of 4 columns).
+__global__ void objective_kernel(const tsenor::ScoreSrc S, const uint32_t* __restrict__ bits_a,
+                                 const uint32_t* __restrict__ bits_b, int64_t rows, int64_t cols, int64_t wpr,
+                                 double* out) {
+    double acc_a = 0.0, acc_b = 0.0;
+    const int64_t qpr = cols / 4, nq = rows * qpr;
+    for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < nq;
          idx += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t r = idx / wpr, wd = idx % wpr;
-        uint32_t m = bits[idx];
-        while (m) {
-            const int b = __ffs(m) - 1;
-            m &= m - 1;
-            const int64_t c = wd * 32 + b;
-            if (c < cols) acc += (double)fabsf(scores[r * ld + c]);
+        const int64_t r = idx / qpr, c = (idx % qpr) * 4;
+        const uint32_t ma = (bits_a[r * wpr + c / 32] >> (c % 32)) & 15u;
+        const uint32_t mb = bits_b ? (bits_b[r * wpr + c / 32] >> (c % 32)) & 15u : 0u;
+        if ((ma | mb) == 0u) continue;
+        const float4 v = tsenor::load_score_quad(S, r, c);
+        const float e[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            if ((ma >> k) & 1u) acc_a += (double)e[k];
+            if ((mb >> k) & 1u) acc_b += (double)e[k];
         }
     }
-    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-    __shared__ double part[32];
+    for (int off = 16; off > 0; off >>= 1) {
+        acc_a += __shfl_xor_sync(0xffffffffu, acc_a, off);
+        acc_b += __shfl_xor_sync(0xffffffffu, acc_b, off);
+    }
+    __shared__ double part[2][32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (lane == 0) part[warp] = acc;
+    if (lane == 0) { part[0][warp] = acc_a; part[1][warp] = acc_b; }
     __syncthreads();
     if (warp == 0) {
-        acc = (lane < (int)(blockDim.x >> 5)) ? part[lane] : 0.0;
-        for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-        if (lane == 0) atomicAdd(out, acc);
+        acc_a = (lane < (int)(blockDim.x >> 5)) ? part[0][lane] : 0.0;
+        acc_b = (lane < (int)(blockDim.x >> 5)) ? part[1][lane] : 0.0;
+        for (int off = 16; off > 0; off >>= 1) {
+            acc_a += __shfl_xor_sync(0xffffffffu, acc_a, off);
+            acc_b += __shfl_xor_sync(0xffffffffu, acc_b, off);
+        }
+        if (lane == 0) {
+            atomicAdd(out, acc_a);
+            if (bits_b) atomicAdd(out + 1, acc_b);
+        }
+    }
+}
+
+// mask_inout <- prev wherever the previous mask retained more score (obj2 = {new, prev}).
+__global__ void keep_better_kernel(const double* __restrict__ obj2, const uint32_t* __restrict__ prev,
+                                   uint32_t* __restrict__ mask_inout, int64_t nwords) {
+    if (!(obj2[0] < obj2[1])) return;
+    for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < nwords;
+         idx += (int64_t)gridDim.x * blockDim.x)
+        mask_inout[idx] = prev[idx];
+}
+
+__global__ void scores_max_kernel(const tsenor::ScoreSrc S, int64_t rows, int64_t cols, unsigned int* out_bits) {
+    float m = 0.f;
+    const int64_t qpr = cols / 4, nq = rows * qpr;
+    for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < nq;
+         idx += (int64_t)gridDim.x * blockDim.x) {
+        const float4 v = tsenor::load_score_quad(S, idx / qpr, (idx % qpr) * 4);
+        m = fmaxf(fmaxf(m, fmaxf(v.x, v.y)), fmaxf(v.z, v.w));  // fmaxf drops NaN
+    }
+    for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+    // non-negative floats order like their bit patterns
+    if ((threadIdx.x & 31) == 0) atomicMax(out_bits, __float_as_uint(m));
+}
+
+__global__ void materialize_kernel(const tsenor::ScoreSrc S, int64_t rows, int64_t cols, float* out,
+                                   int64_t ld_out) {
+    const int64_t qpr = cols / 4, nq = rows * qpr;
+    for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < nq;
+         idx += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = idx / qpr, c = (idx % qpr) * 4;
+        const float4 v = tsenor::load_score_quad(S, r, c);
+        float* p = out + r * ld_out + c;
+        p[0] = v.x; p[1] = v.y; p[2] = v.z; p[3] = v.w;
+    }
+}
+
+// "Simple" rounding: one warp per block; lane i is row i in the first pass and column i in
+// the second.  Ranks by counting under the strict order (key descending, index ascending).
+__device__ __forceinline__ bool key_before(float ka, int ia, float kb, int ib) {
+    return ka > kb || (ka == kb && ia < ib);
+}
+__global__ void simple_round_kernel(const float* __restrict__ key, int64_t ld, int64_t rows, int64_t cols,
+                                    int64_t wpr, int N, int M, uint32_t* bits) {
+    __shared__ float ks[4][32][33];
+    __shared__ unsigned rowmask[4][32];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t nbc = cols / M, nblk = (rows / M) * nbc;
+    for (int64_t b = blockIdx.x * 4LL + warp; b < nblk; b += gridDim.x * 4LL) {
+        const int64_t r0 = (b / nbc) * M, c0 = (b % nbc) * M;
+        for (int i = 0; i < M; ++i)
+            if (lane < M) {
+                float k = key[(r0 + i) * ld + c0 + lane];
+                if (!(k == k)) k = __int_as_float(0xff800000);
+                ks[warp][i][lane] = k + 0.0f;
+            }
+        __syncwarp();
+        unsigned keep = 0u;
+        if (lane < M) {   // row pass: the N best of my row
+            for (int j = 0; j < M; ++j) {
+                int rank = 0;
+                for (int j2 = 0; j2 < M; ++j2) rank += key_before(ks[warp][lane][j2], j2, ks[warp][lane][j], j) ? 1 : 0;
+                if (rank < N) keep |= 1u << j;
+            }
+        }
+        rowmask[warp][lane] = keep;
+        __syncwarp();
+        unsigned colkeep = 0u;   // bits over rows, for my column
+        if (lane < M) {
+            unsigned surv = 0u;
+            for (int i = 0; i < M; ++i) surv |= ((rowmask[warp][i] >> lane) & 1u) << i;
+            for (int i = 0; i < M; ++i) {
+                if (!((surv >> i) & 1u)) continue;
+                int rank = 0;
+                for (int i2 = 0; i2 < M; ++i2)
+                    if ((surv >> i2) & 1u) rank += key_before(ks[warp][i2][lane], i2, ks[warp][i][lane], i) ? 1 : 0;
+                if (rank < N) colkeep |= 1u << i;
+            }
+        }
+        __syncwarp();
+        rowmask[warp][lane] = colkeep;   // now indexed by column
+        __syncwarp();
+        if (lane < M) {
+            unsigned row = 0u;
+            for (int j = 0; j < M; ++j) row |= ((rowmask[warp][j] >> lane) & 1u) << j;
+            if (row) atomicOr(&bits[(r0 + lane) * wpr + c0 / 32], row << (c0 % 32));
+        }
+        __syncwarp();
     }
 }
 
@@ -149,20 +289,6 @@ __global__ void check_kernel(const uint32_t* __restrict__ bits, int64_t rows, in
     if ((threadIdx.x & 31) == 0 && bad) atomicAdd(bad_out, bad);
 }
 
-__global__ void max_abs_kernel(const float* __restrict__ scores, int64_t rows, int64_t cols, int64_t ld,
-                               unsigned int* out_bits) {
-    float m = 0.f;
-    const int64_t n = rows * cols;
-    for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < n;
-         idx += (int64_t)gridDim.x * blockDim.x) {
-        const float v = fabsf(scores[(idx / cols) * ld + idx % cols]);
-        m = fmaxf(m, v);  // fmaxf drops NaN
-    }
-    for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-    // non-negative floats order like their bit patterns
-    if ((threadIdx.x & 31) == 0) atomicMax(out_bits, __float_as_uint(m));
-}
-
 int grid_for(int64_t work, int threads) {
     int64_t g = (work + threads - 1) / threads;
     if (g < 1) g = 1;
@@ -181,6 +307,20 @@ int trivial_mask(uint32_t* bits, int64_t rows, int64_t cols, bool ones, cudaStre
 
 extern "C" {
 
+static int solve_on(const tsenor::ScoreSrc& src, int64_t rows, int64_t cols, int N, int M, float tau, int iters,
+                    int ls_steps, uint32_t* mask_bits_out, int32_t* dev_status, cudaStream_t st) {
+    if (N == 0 || N == M) return trivial_mask(mask_bits_out, rows, cols, N == M, st);
+    tsenor::Params P{};
+    P.src = src;
+    P.bits = mask_bits_out; P.wpr = (cols + 31) / 32;
+    P.rows = rows; P.cols = cols;
+    P.N = N; P.Nf = (float)N; P.log2N = (float)std::log2((double)N);
+    set_tau(P, tau);
+    P.iters = iters; P.ls_steps = ls_steps;
+    P.status = dev_status;
+    return dispatch<0>(P, M, st);
+}
+
 int tsenor_solve(const float* scores, int64_t rows, int64_t cols, int64_t ld, int N, int M, float tau, int iters,
                  int ls_steps, uint32_t* mask_bits_out, int32_t* dev_status, tsenor_stream_t stream) {
     if (!valid_M(M) || N < 0 || N > M) return TSENOR_ERR_NM;
@@ -188,18 +328,82 @@ int tsenor_solve(const float* scores, int64_t rows, int64_t cols, int64_t ld, in
     if (iters < 0 || !(tau >= 0.0f) || !std::isfinite(tau)) return TSENOR_ERR_ARG;
     if (rows == 0 || cols == 0) return TSENOR_OK;
     if (!scores || !mask_bits_out) return TSENOR_ERR_NULL;
+    return solve_on(abs_source(scores, ld), rows, cols, N, M, tau, iters, ls_steps, mask_bits_out, dev_status,
+                    (cudaStream_t)stream);
+}
+
+int tsenor_solve_scores(const tsenor_scores_t* s, int64_t rows, int64_t cols, int N, int M, float tau, int iters,
+                        int ls_steps, uint32_t* mask_bits_out, int32_t* dev_status, tsenor_stream_t stream) {
+    if (!valid_M(M) || N < 0 || N > M) return TSENOR_ERR_NM;
+    if (int rc = check_matrix(rows, cols, cols, M)) return rc;
+    if (iters < 0 || !(tau >= 0.0f) || !std::isfinite(tau)) return TSENOR_ERR_ARG;
+    tsenor::ScoreSrc src{};
+    if (int rc = make_source(s, cols, &src)) return rc;
+    if (rows == 0 || cols == 0) return TSENOR_OK;
+    if (!mask_bits_out) return TSENOR_ERR_NULL;
+    return solve_on(src, rows, cols, N, M, tau, iters, ls_steps, mask_bits_out, dev_status, (cudaStream_t)stream);
+}
+
+static int max_on(const tsenor::ScoreSrc& src, int64_t rows, int64_t cols, float* dev_max_out, cudaStream_t st) {
+    if (cudaMemsetAsync(dev_max_out, 0, sizeof(float), st) != cudaSuccess) return finish_launch(), TSENOR_ERR_CUDA;
+    if (rows == 0 || cols == 0) return TSENOR_OK;
+    scores_max_kernel<<<grid_for(rows * (cols / 4), 256 * 2), 256, 0, st>>>(
+        src, rows, cols, reinterpret_cast<unsigned int*>(dev_max_out));
+    return finish_launch();
+}
+
+int tsenor_scores_max(const tsenor_scores_t* s, int64_t rows, int64_t cols, float* dev_max_out,
+                      tsenor_stream_t stream) {
+    if (rows < 0 || cols < 0 || cols % 4) return TSENOR_ERR_SHAPE;
+    tsenor::ScoreSrc src{};
+    if (int rc = make_source(s, cols, &src)) return rc;
+    if (!dev_max_out) return TSENOR_ERR_NULL;
+    return max_on(src, rows, cols, dev_max_out, (cudaStream_t)stream);
+}
+
+int tsenor_scores_materialize(const tsenor_scores_t* s, int64_t rows, int64_t cols, float* scores_out,
+                              int64_t ld_out, tsenor_stream_t stream) {
+    if (rows < 0 || cols < 0 || cols % 4 || ld_out < cols) return TSENOR_ERR_SHAPE;
+    tsenor::ScoreSrc src{};
+    if (int rc = make_source(s, cols, &src)) return rc;
+    if (rows == 0 || cols == 0) return TSENOR_OK;
+    if (!scores_out) return TSENOR_ERR_NULL;
+    materialize_kernel<<<grid_for(rows * (cols / 4), 256), 256, 0, (cudaStream_t)stream>>>(src, rows, cols,
+                                                                                          scores_out, ld_out);
+    return finish_launch();
+}
+
+int tsenor_keep_better(const tsenor_scores_t* s, int64_t rows, int64_t cols, const uint32_t* prev_mask,
+                       uint32_t* mask_inout, double* dev_obj2_out, tsenor_stream_t stream) {
+    if (rows < 0 || cols < 0 || cols % 4) return TSENOR_ERR_SHAPE;
+    tsenor::ScoreSrc src{};
+    if (int rc = make_source(s, cols, &src)) return rc;
+    if (!dev_obj2_out) return TSENOR_ERR_NULL;
     cudaStream_t st = (cudaStream_t)stream;
-    if (N == 0 || N == M) return trivial_mask(mask_bits_out, rows, cols, N == M, st);
-    tsenor::Params P{};
-    P.scores = scores; P.ld = ld;
-    P.bits = mask_bits_out; P.wpr = (cols + 31) / 32;
-    P.rows = rows; P.cols = cols;
-    P.N = N; P.Nf = (float)N; P.log2N = (float)std::log2((double)N);
-    set_tau(P, tau);
-    P.iters = iters; P.ls_steps = ls_steps;
-    P.status = dev_status;
-    P.vec_scores = aligned16(scores, ld);
-    return dispatch<0>(P, M, st);
+    if (cudaMemsetAsync(dev_obj2_out, 0, 2 * sizeof(double), st) != cudaSuccess)
+        return finish_launch(), TSENOR_ERR_CUDA;
+    if (rows == 0 || cols == 0) return TSENOR_OK;
+    if (!prev_mask || !mask_inout) return TSENOR_ERR_NULL;
+    const int64_t wpr = (cols + 31) / 32;
+    objective_kernel<<<grid_for(rows * (cols / 4), 256), 256, 0, st>>>(src, mask_inout, prev_mask, rows, cols, wpr,
+                                                                      dev_obj2_out);
+    if (int rc = finish_launch()) return rc;
+    keep_better_kernel<<<grid_for(rows * wpr, 256), 256, 0, st>>>(dev_obj2_out, prev_mask, mask_inout, rows * wpr);
+    return finish_launch();
+}
+
+int tsenor_simple_round(const float* plan_key, int64_t ld_plan, int64_t rows, int64_t cols, int N, int M,
+                        uint32_t* mask_bits_out, tsenor_stream_t stream) {
+    if (!valid_M(M) || N < 1 || N >= M) return TSENOR_ERR_NM;
+    if (int rc = check_matrix(rows, cols, ld_plan, M)) return rc;
+    if (rows == 0 || cols == 0) return TSENOR_OK;
+    if (!plan_key || !mask_bits_out) return TSENOR_ERR_NULL;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int64_t wpr = (cols + 31) / 32, nblk = (rows / M) * (cols / M);
+    if (cudaMemsetAsync(mask_bits_out, 0, sizeof(uint32_t) * (size_t)(rows * wpr), st) != cudaSuccess)
+        return finish_launch(), TSENOR_ERR_CUDA;
+    simple_round_kernel<<<grid_for(nblk, 4), 128, 0, st>>>(plan_key, ld_plan, rows, cols, wpr, N, M, mask_bits_out);
+    return finish_launch();
 }
 
 int tsenor_dykstra(const float* scores, int64_t rows, int64_t cols, int64_t ld, int N, int M, float tau, int iters,
@@ -211,14 +415,13 @@ int tsenor_dykstra(const float* scores, int64_t rows, int64_t cols, int64_t ld, 
     if (rows == 0 || cols == 0) return TSENOR_OK;
     if (!scores || !plan_out) return TSENOR_ERR_NULL;
     tsenor::Params P{};
-    P.scores = scores; P.ld = ld;
+    P.src = abs_source(scores, ld);
     P.plan = plan_out; P.ld_plan = ld_plan; P.plan_is_log = plan_is_log;
     P.rows = rows; P.cols = cols;
     P.N = N; P.Nf = (float)N; P.log2N = (float)std::log2((double)N);
     set_tau(P, tau);
     P.iters = iters; P.ls_steps = -1;
     P.status = dev_status;
-    P.vec_scores = aligned16(scores, ld);
     return dispatch<1>(P, M, (cudaStream_t)stream);
 }
 
@@ -233,28 +436,28 @@ int tsenor_round(const float* plan_key, int64_t ld_plan, const float* scores, in
     cudaStream_t st = (cudaStream_t)stream;
     if (N == 0 || N == M) return trivial_mask(mask_bits_out, rows, cols, N == M, st);
     tsenor::Params P{};
-    P.scores = scores; P.ld = ld;
+    P.src = abs_source(scores, ld);
     P.keys = plan_key; P.ld_keys = ld_plan;
     P.bits = mask_bits_out; P.wpr = (cols + 31) / 32;
     P.rows = rows; P.cols = cols;
     P.N = N; P.Nf = (float)N; P.log2N = 0.f;
     P.iters = 0; P.ls_steps = ls_steps;
     P.status = dev_status;
-    P.vec_scores = aligned16(scores, ld);
     P.vec_keys = aligned16(plan_key, ld_plan);
     return dispatch<2>(P, M, st);
 }
 
 int tsenor_objective(const float* scores, int64_t ld, const uint32_t* mask_bits, int64_t rows, int64_t cols,
                      double* dev_sum_out, tsenor_stream_t stream) {
-    if (rows < 0 || cols < 0 || ld < cols) return TSENOR_ERR_SHAPE;
+    if (rows < 0 || cols < 0 || ld < cols || cols % 4) return TSENOR_ERR_SHAPE;
     if (!dev_sum_out) return TSENOR_ERR_NULL;
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemsetAsync(dev_sum_out, 0, sizeof(double), st) != cudaSuccess) return finish_launch(), TSENOR_ERR_CUDA;
     if (rows == 0 || cols == 0) return TSENOR_OK;
     if (!scores || !mask_bits) return TSENOR_ERR_NULL;
     const int64_t wpr = (cols + 31) / 32;
-    objective_kernel<<<grid_for(rows * wpr, 256), 256, 0, st>>>(scores, ld, mask_bits, rows, cols, wpr, dev_sum_out);
+    objective_kernel<<<grid_for(rows * (cols / 4), 256), 256, 0, st>>>(abs_source(scores, ld), mask_bits, nullptr,
+                                                                      rows, cols, wpr, dev_sum_out);
     return finish_launch();
 }
 
@@ -276,15 +479,10 @@ int tsenor_check(const uint32_t* mask_bits, int64_t rows, int64_t cols, int N, i
 
 int tsenor_max_abs(const float* scores, int64_t rows, int64_t cols, int64_t ld, float* dev_max_out,
                    tsenor_stream_t stream) {
-    if (rows < 0 || cols < 0 || ld < cols) return TSENOR_ERR_SHAPE;
+    if (rows < 0 || cols < 0 || ld < cols || cols % 4) return TSENOR_ERR_SHAPE;
     if (!dev_max_out) return TSENOR_ERR_NULL;
-    cudaStream_t st = (cudaStream_t)stream;
-    if (cudaMemsetAsync(dev_max_out, 0, sizeof(float), st) != cudaSuccess) return finish_launch(), TSENOR_ERR_CUDA;
-    if (rows == 0 || cols == 0) return TSENOR_OK;
-    if (!scores) return TSENOR_ERR_NULL;
-    max_abs_kernel<<<grid_for(rows * cols, 256 * 8), 256, 0, st>>>(scores, rows, cols, ld,
-                                                                   reinterpret_cast<unsigned int*>(dev_max_out));
-    return finish_launch();
+    if (rows > 0 && cols > 0 && !scores) return TSENOR_ERR_NULL;
+    return max_on(abs_source(scores, ld), rows, cols, dev_max_out, (cudaStream_t)stream);
 }
 
 int64_t tsenor_mask_words_per_row(int64_t cols) { return cols <= 0 ? 0 : (cols + 31) / 32; }
@@ -293,7 +491,7 @@ const char* tsenor_strerror(int status) {
     switch (status) {
         case TSENOR_OK: return "ok";
         case TSENOR_ERR_NULL: return "a required pointer is NULL";
-        case TSENOR_ERR_SHAPE: return "bad shape: negative size, ld < cols, or rows/cols not a multiple of M";
+        case TSENOR_ERR_SHAPE: return "bad shape: negative size, ld < cols, or rows/cols not a multiple of M (of 4)";
         case TSENOR_ERR_NM: return "bad N:M: M must be 4, 8, 16 or 32 and N within range";
         case TSENOR_ERR_ARG: return "bad argument: iters < 0 or tau negative / not finite";
         case TSENOR_ERR_CUDA: return "CUDA launch failed: see tsenor_last_cuda_error()";

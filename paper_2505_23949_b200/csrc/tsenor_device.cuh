@@ -360,13 +360,78 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>:
 }
 
 // ---------------------------------------------------------------------------
-// Panel loader: |score| of an M x PANEL panel into shared memory, coalesced,
-// 16-byte vector loads when the addresses allow it.  Returns non-zero if a
-// non-finite value was seen by this thread.
+// Score source: the matrix the solver works on, described rather than
+// materialised (Section 4: magnitude, ADMM D-update, SparseGPT group, Wanda).
+// One fp32 rounding per operation, no fused multiply-add.
+// ---------------------------------------------------------------------------
+enum : int { SC_ABS = 0, SC_ADMM = 1, SC_COLDIV = 2, SC_COLMUL = 3 };
+
+struct ScoreSrc {
+    int kind, w_is_bf16;
+    const void* w; int64_t ld;
+    const float* v; int64_t ld_v;
+    float scalar;
+    const float* colvec;
+    int vec_w, vec_v, vec_c;       // 16-byte (8-byte for bf16) vector loads allowed
+};
+
+__device__ __forceinline__ float score_of(int kind, float w, float v, float scalar, float cv) {
+    switch (kind) {
+        case SC_ADMM: { const float s = __fadd_rn(w, __fmul_rn(v, scalar)); return __fmul_rn(s, s); }
+        case SC_COLDIV: return fabsf(__fdiv_rn(w, cv));
+        case SC_COLMUL: return __fmul_rn(fabsf(w), cv);
+        default: return fabsf(w);
+    }
+}
+
+// Scores of the four consecutive elements (r, c .. c+3); c is a multiple of 4.
+__device__ __forceinline__ float4 load_score_quad(const ScoreSrc& S, int64_t r, int64_t c) {
+    float4 w;
+    if (S.w_is_bf16) {
+        const unsigned short* p = static_cast<const unsigned short*>(S.w) + r * S.ld + c;
+        unsigned lo, hi;
+        if (S.vec_w) {
+            const uint2 q = __ldg(reinterpret_cast<const uint2*>(p));
+            lo = q.x; hi = q.y;
+        } else {
+            lo = __ldg(p) | ((unsigned)__ldg(p + 1) << 16);
+            hi = __ldg(p + 2) | ((unsigned)__ldg(p + 3) << 16);
+        }
+        w = make_float4(__uint_as_float(lo << 16), __uint_as_float(lo & 0xffff0000u),
+                        __uint_as_float(hi << 16), __uint_as_float(hi & 0xffff0000u));
+    } else {
+        const float* p = static_cast<const float*>(S.w) + r * S.ld + c;
+        if (S.vec_w) w = __ldg(reinterpret_cast<const float4*>(p));
+        else w = make_float4(__ldg(p), __ldg(p + 1), __ldg(p + 2), __ldg(p + 3));
+    }
+    if (S.kind == SC_ABS) return make_float4(fabsf(w.x), fabsf(w.y), fabsf(w.z), fabsf(w.w));
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f), cv = make_float4(1.f, 1.f, 1.f, 1.f);
+    if (S.kind == SC_ADMM) {
+        const float* p = S.v + r * S.ld_v + c;
+        if (S.vec_v) v = __ldg(reinterpret_cast<const float4*>(p));
+        else v = make_float4(__ldg(p), __ldg(p + 1), __ldg(p + 2), __ldg(p + 3));
+    } else {
+        const float* p = S.colvec + c;
+        if (S.vec_c) cv = __ldg(reinterpret_cast<const float4*>(p));
+        else cv = make_float4(__ldg(p), __ldg(p + 1), __ldg(p + 2), __ldg(p + 3));
+    }
+    return make_float4(score_of(S.kind, w.x, v.x, S.scalar, cv.x), score_of(S.kind, w.y, v.y, S.scalar, cv.y),
+                       score_of(S.kind, w.z, v.z, S.scalar, cv.z), score_of(S.kind, w.w, v.w, S.scalar, cv.w));
+}
+
+__device__ __forceinline__ int any_nonfinite(const float4& v) {
+    return !(fabsf(v.x) <= 3.4028234e38f) | !(fabsf(v.y) <= 3.4028234e38f) |
+           !(fabsf(v.z) <= 3.4028234e38f) | !(fabsf(v.w) <= 3.4028234e38f);
+}
+
+// ---------------------------------------------------------------------------
+// Panel loaders: an M x PANEL panel into shared memory, coalesced, vector
+// loads when the addresses allow it.  Return non-zero if a non-finite value
+// was seen by this thread.
 // ---------------------------------------------------------------------------
 template <int M>
-__device__ __forceinline__ int load_panel(const float* __restrict__ src, int64_t ld, int64_t r0, int64_t c0,
-                                          int64_t cols, bool vec_ok, bool take_abs, float* __restrict__ dst) {
+__device__ __forceinline__ int load_score_panel(const ScoreSrc& S, int64_t r0, int64_t c0, int64_t cols,
+                                                float* __restrict__ dst) {
     using G = Geom<M>;
     constexpr int V = G::PANEL / 4;
     int bad = 0;
@@ -374,17 +439,30 @@ __device__ __forceinline__ int load_panel(const float* __restrict__ src, int64_t
         const int r = idx / V, c = (idx % V) * 4;
         const int64_t gc = c0 + c;
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (gc < cols) {  // cols is a multiple of 4, so a quad is all in or all out
+        if (gc < cols) v = load_score_quad(S, r0 + r, gc);  // cols % 4 == 0: a quad is all in or all out
+        bad |= any_nonfinite(v);
+        float* d = dst + r * G::WS + c;
+        d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
+    }
+    return bad;
+}
+
+template <int M>
+__device__ __forceinline__ int load_key_panel(const float* __restrict__ src, int64_t ld, int64_t r0, int64_t c0,
+                                              int64_t cols, bool vec_ok, float* __restrict__ dst) {
+    using G = Geom<M>;
+    constexpr int V = G::PANEL / 4;
+    int bad = 0;
+    for (int idx = threadIdx.x; idx < M * V; idx += WARPS * 32) {
+        const int r = idx / V, c = (idx % V) * 4;
+        const int64_t gc = c0 + c;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (gc < cols) {
             const float* p = src + (r0 + r) * ld + gc;
-            if (vec_ok) {
-                v = __ldg(reinterpret_cast<const float4*>(p));
-            } else {
-                v.x = __ldg(p); v.y = __ldg(p + 1); v.z = __ldg(p + 2); v.w = __ldg(p + 3);
-            }
+            if (vec_ok) v = __ldg(reinterpret_cast<const float4*>(p));
+            else v = make_float4(__ldg(p), __ldg(p + 1), __ldg(p + 2), __ldg(p + 3));
         }
-        if (take_abs) { v.x = fabsf(v.x); v.y = fabsf(v.y); v.z = fabsf(v.z); v.w = fabsf(v.w); }
-        bad |= !(fabsf(v.x) <= 3.4028234e38f) | !(fabsf(v.y) <= 3.4028234e38f) |
-               !(fabsf(v.z) <= 3.4028234e38f) | !(fabsf(v.w) <= 3.4028234e38f);
+        bad |= any_nonfinite(v);
         float* d = dst + r * G::WS + c;
         d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
     }
@@ -615,7 +693,7 @@ __device__ __forceinline__ unsigned round_block(float* ks, const float* ws, Roun
 // 2: Algorithm 2 only (keys from global).
 // ---------------------------------------------------------------------------
 struct Params {
-    const float* scores; int64_t ld;
+    ScoreSrc src;
     const float* keys;   int64_t ld_keys;
     float* plan;         int64_t ld_plan; int plan_is_log;
     uint32_t* bits;      int64_t wpr;
@@ -625,7 +703,7 @@ struct Params {
     float c_hi, c_lo;              // tau * log2(e), split in two floats
     int iters, ls_steps;
     int32_t* status;
-    int vec_scores, vec_keys;
+    int vec_keys;
 };
 
 template <int M, int MODE> struct SmemLayout {
@@ -661,9 +739,9 @@ __global__ void __launch_bounds__(WARPS * 32, MinBlocks<M>::value) tsenor_kernel
     int flags = 0;
 
     // ---- block loader
-    if (load_panel<M>(P.scores, P.ld, r0, c0, P.cols, P.vec_scores != 0, true, sm.w)) flags |= DEV_NONFINITE;
+    if (load_score_panel<M>(P.src, r0, c0, P.cols, sm.w)) flags |= DEV_NONFINITE;
     if (MODE == 2)
-        if (load_panel<M>(P.keys, P.ld_keys, r0, c0, P.cols, P.vec_keys != 0, false, sm.k)) flags |= DEV_NONFINITE;
+        if (load_key_panel<M>(P.keys, P.ld_keys, r0, c0, P.cols, P.vec_keys != 0, sm.k)) flags |= DEV_NONFINITE;
     if (MODE != 1)
         for (int idx = threadIdx.x; idx < M * G::WORDS; idx += WARPS * 32) sm.bits[idx] = 0u;
     __syncthreads();

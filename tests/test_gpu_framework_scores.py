@@ -1,0 +1,133 @@
+"""GPU parity of the framework score sources (magnitude, ADMM D-update, SparseGPT group,
+Wanda), the mask safeguard and the simple rounding, against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2505_23949_b200 import binding as ts
+from paper_2505_23949_b200 import synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
+
+
+def _bits(t):
+    return t.cpu().numpy().view(np.uint32)
+
+
+def _sources(rows, cols, seed):
+    """(name, binding Scores, oracle fp32 score matrix) for every kind."""
+    rng = np.random.default_rng(seed)
+    W = (rng.standard_normal((rows, cols)) * 0.02).astype(np.float32)
+    V = (rng.standard_normal((rows, cols)) * 0.01).astype(np.float32)
+    d = (np.abs(rng.standard_normal(cols)) + 0.05).astype(np.float32)
+    a = rng.lognormal(0.0, 1.0, cols).astype(np.float32)
+    Wb = torch.from_numpy(W).to(torch.bfloat16)
+    Wb32 = Wb.to(torch.float32).numpy()
+    Wd, Vd, dd, ad = _dev(W), _dev(V), _dev(d), _dev(a)
+    return [
+        ("abs", ts.Scores(ts.SCORES_ABS, Wd), oracle.scores(oracle.SCORES_ABS, W)),
+        ("admm", ts.Scores(ts.SCORES_ADMM, Wd, v=Vd, scalar=1 / 3.0), oracle.scores(oracle.SCORES_ADMM, W, V, np.float32(1 / 3.0))),
+        ("coldiv", ts.Scores(ts.SCORES_COLDIV, Wd, colvec=dd), oracle.scores(oracle.SCORES_COLDIV, W, colvec=d)),
+        ("colmul", ts.Scores(ts.SCORES_COLMUL, Wd, colvec=ad), oracle.scores(oracle.SCORES_COLMUL, W, colvec=a)),
+        ("colmul_bf16", ts.Scores(ts.SCORES_COLMUL, Wb.to(DEV), colvec=ad), oracle.scores(oracle.SCORES_COLMUL, Wb32, colvec=a)),
+    ]
+
+
+@pytest.mark.parametrize("M,N,rows,cols", [(32, 16, 64, 352), (16, 8, 32, 592), (8, 4, 24, 1096), (4, 2, 16, 1060)])
+def test_described_scores_are_bit_exact_and_solve_like_materialised_ones(M, N, rows, cols):
+    for name, src, ref in _sources(rows, cols, 7 * M + N):
+        got = ts.scores_materialize(src).cpu().numpy()
+        assert np.array_equal(got, ref), name                       # same fp32 bits as the oracle
+        assert float(ts.scores_max(src).item()) == float(ref.max()), name
+        tau = synth.default_tau(ref.max())
+        st = ts.new_status(DEV)
+        mask = _bits(ts.solve_scores(src, N, M, tau, 300, status=st))
+        assert int(st.item()) == 0
+        assert np.array_equal(mask, _bits(ts.solve(_dev(ref), N, M, tau, 300))), name
+        assert oracle.count_infeasible(mask, rows, cols, N, M) == 0
+        want = oracle.solve(ref, N, M, tau, 300)
+        o_gpu, o_ref = oracle.objective(ref, mask), oracle.objective(ref, want)
+        assert abs(o_gpu - o_ref) <= 1e-4 * o_ref, name
+
+
+def test_unaligned_and_strided_sources():
+    rng = np.random.default_rng(5)
+    big = (rng.standard_normal((40, 300)) * 0.02).astype(np.float32)
+    bigd = _dev(big)
+    a = rng.lognormal(0, 1, 264).astype(np.float32)
+    buf = torch.zeros(265, device=DEV)
+    buf[1:] = _dev(a)
+    wv = bigd[1:33, 3:267]                                          # ld 300, odd offset
+    src = ts.Scores(ts.SCORES_COLMUL, wv, colvec=buf[1:])
+    ref = oracle.scores(oracle.SCORES_COLMUL, big[1:33, 3:267], colvec=a)
+    assert np.array_equal(ts.scores_materialize(src).cpu().numpy(), ref)
+    wb = torch.from_numpy(big).to(torch.bfloat16).to(DEV)[1:33, 3:267]
+    srcb = ts.Scores(ts.SCORES_COLMUL, wb, colvec=buf[1:])
+    refb = oracle.scores(oracle.SCORES_COLMUL, wb.to(torch.float32).cpu().numpy(), colvec=a)
+    assert np.array_equal(ts.scores_materialize(srcb).cpu().numpy(), refb)
+    m = _bits(ts.solve_scores(srcb, 4, 8, synth.default_tau(refb.max()), 100))
+    assert oracle.count_infeasible(m, 32, 264, 4, 8) == 0
+
+
+def test_admm_sequence_with_safeguard_matches_oracle():
+    """A short ADMM-like sequence: the score matrix drifts, every iteration solves and keeps
+    the previous mask if the new one retains less (Appendix A.1.3)."""
+    rng = np.random.default_rng(9)
+    M, N, rows, cols = 16, 8, 64, 512
+    W = (rng.standard_normal((rows, cols)) * 0.02).astype(np.float32)
+    Wd = _dev(W)
+    prev_gpu = prev_ref = None
+    for t in range(5):
+        V = ((0.2 * t) * rng.standard_normal((rows, cols)) * 0.02).astype(np.float32)
+        rho = np.float32(1.0 / (0.5 + 0.3 * t))
+        src = ts.Scores(ts.SCORES_ADMM, Wd, v=_dev(V), scalar=float(rho))
+        sc = oracle.scores(oracle.SCORES_ADMM, W, V, rho)
+        tau = float(200.0 / ts.scores_max(src).item())
+        new_gpu = ts.solve_scores(src, N, M, tau, 120)
+        if t == 3:                                                  # a deliberately poor candidate
+            new_gpu = ts.round_plan(-ts.scores_materialize(src), ts.scores_materialize(src), N, M)
+        if prev_gpu is None:
+            prev_gpu = new_gpu
+            continue
+        cand = _bits(new_gpu).copy()
+        obj2 = ts.keep_better(src, prev_gpu, new_gpu).cpu().numpy()
+        kept_ref, o_new, o_prev = oracle.keep_better(sc, _bits(prev_gpu), cand)
+        assert np.array_equal(_bits(new_gpu), kept_ref)
+        assert abs(obj2[0] - o_new) <= 1e-12 * o_new and abs(obj2[1] - o_prev) <= 1e-12 * o_prev
+        if t == 3:
+            assert o_new < o_prev and np.array_equal(_bits(new_gpu), _bits(prev_gpu))
+        prev_gpu = new_gpu
+
+
+@pytest.mark.parametrize("M,N", [(4, 2), (8, 4), (16, 8), (32, 16), (8, 3), (32, 5)])
+def test_simple_rounding_is_bit_exact(M, N):
+    rng = np.random.default_rng(M * 10 + N)
+    rows, cols = 2 * M, 10 * M + (32 if M < 32 else 0)
+    W = synth.gaussian_abs(rows, cols, 0.02, M + N)
+    tau = synth.default_tau(W.max())
+    x = ts.dykstra(_dev(W), N, M, tau, 300, plan_is_log=True)
+    for key in (x.cpu().numpy(), np.round(rng.standard_normal((rows, cols)) * 2).astype(np.float32)):
+        got = _bits(ts.simple_round(_dev(key), N, M))
+        assert np.array_equal(got, oracle.simple_round(key, N, M))
+
+
+def test_descriptor_errors():
+    W = _dev(np.zeros((8, 16), np.float32))
+    src = ts.Scores(ts.SCORES_ADMM, W, v=W, scalar=float("nan"))
+    with pytest.raises(ts.TsenorError) as e:
+        ts.solve_scores(src, 2, 4, 1.0)
+    assert e.value.status == ts.ERR_ARG
+    bad = ts.Scores(ts.SCORES_COLDIV, W)                            # colvec missing
+    with pytest.raises(ts.TsenorError) as e:
+        ts.scores_max(bad)
+    assert e.value.status == ts.ERR_NULL
+    bf = ts.Scores(ts.SCORES_ABS, W.to(torch.bfloat16))             # bf16 only with COLMUL
+    with pytest.raises(ts.TsenorError) as e:
+        ts.scores_materialize(bf)
+    assert e.value.status == ts.ERR_ARG
