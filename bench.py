@@ -8,7 +8,9 @@ down-projection score matrix (2 x 57,344 blocks of 32x32), Student-t(3)
 scores, tau = 200 / max|W| per matrix.
 
 Prints ONE JSON line (rank 0).  ``--impl reference`` times the CPU oracle on a
-bounded sample of the same workload instead.
+bounded sample of the same workload instead.  ``--workload`` selects one of the
+other configurations (0, 1, 2, 3, 5) or loader modes (admm, wanda); the default
+is the headline above.
 """
 import argparse
 import json
