@@ -234,3 +234,29 @@ def test_non_finite_scores_are_flagged_and_nothing_hangs():
     keep[8:16, 2] = False     # block (1,8) holds the inf  -> word 2 rows 8..15
     assert np.array_equal(got[keep], ref[keep])
     assert np.array_equal(got[0:8, 0] >> 8, ref[0:8, 0] >> 8)
+
+
+@pytest.mark.parametrize("M,N", [(4, 2), (8, 4), (16, 8), (32, 16)])
+def test_degenerate_score_matrices(M, N):
+    """All-equal scores (every key ties: the index order decides everything), all-zero scores,
+    and a single dominant entry per block (tau |w| = 200 against 0 elsewhere)."""
+    rows, cols = 2 * M, 6 * M + 32
+    const = np.full((rows, cols), 0.37, np.float32)
+    zero = np.zeros((rows, cols), np.float32)
+    spike = np.full((rows, cols), 1e-3, np.float32)
+    spike[::M, ::M] = 5.0
+    ramp = (np.arange(rows * cols, dtype=np.float32).reshape(rows, cols) % 7) * 0.1   # few distinct values
+    for W, tau in ((const, 200.0 / 0.37), (zero, 1.0), (spike, 40.0), (ramp, 200.0 / 0.6)):
+        st = ts.new_status(DEV)
+        got = _bits(ts.solve(_dev(W), N, M, tau, 300, status=st))
+        assert int(st.item()) == 0
+        assert oracle.count_infeasible(got, rows, cols, N, M) == 0
+        want = oracle.solve(W, N, M, tau, 300)
+        o_gpu, o_ref = oracle.objective(W, got), oracle.objective(W, want)
+        assert abs(o_gpu - o_ref) <= OBJ_RTOL * max(o_ref, 1e-30)
+        plan = ts.dykstra(_dev(W), N, M, tau, 300).cpu().numpy()
+        assert np.abs(plan - oracle.dykstra(W, N, M, tau, 300)).max() <= PLAN_TOL
+    # with every key equal the mask is decided by the index tie-break alone: identical to the oracle
+    assert np.array_equal(_bits(ts.solve(_dev(const), N, M, 200.0 / 0.37, 300)),
+                          oracle.solve(const, N, M, 200.0 / 0.37, 300))
+    assert np.array_equal(_bits(ts.solve(_dev(zero), N, M, 1.0, 300)), oracle.solve(zero, N, M, 1.0, 300))
