@@ -148,12 +148,12 @@ enum {
                                  colvec_j = [H^-1]_jj (the printed -W/[H^-1]_jj,
                                  magnitude taken)                                      */
     TSENOR_SCORES_COLMUL = 3  /* |W_ij| * colvec_j            Wanda score, colvec_j =
-                                 norm of input feature j; W may be bf16               */
+                                 norm of input feature j                              */
 };
 
 typedef struct tsenor_scores {
     int kind;            /* one of TSENOR_SCORES_*                                     */
-    int w_is_bf16;       /* non-zero: w points to bf16 (only with TSENOR_SCORES_COLMUL) */
+    int w_is_bf16;       /* non-zero: w points to bf16 (widened exactly to fp32), any kind */
     const void *w;       /* rows x cols weights, row-major, leading dimension ld       */
     int64_t ld;
     const float *v;      /* TSENOR_SCORES_ADMM: dual variable V, rows x cols fp32      */

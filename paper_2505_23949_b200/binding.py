@@ -191,7 +191,7 @@ def max_abs(scores, out=None, stream=None):
 class Scores:
     """A described score matrix (``tsenor_scores_t``): keeps the tensors alive and builds
     the descriptor.  kind: SCORES_ABS |W|, SCORES_ADMM (W + V*scalar)^2, SCORES_COLDIV
-    |W / colvec_j|, SCORES_COLMUL |W| * colvec_j (W may be bfloat16)."""
+    |W / colvec_j|, SCORES_COLMUL |W| * colvec_j.  W may be float32 or bfloat16."""
 
     def __init__(self, kind, w, v=None, scalar=0.0, colvec=None):
         if not (isinstance(w, torch.Tensor) and w.is_cuda and w.dim() == 2 and w.stride(1) == 1):

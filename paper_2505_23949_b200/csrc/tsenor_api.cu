@@ -46,7 +46,6 @@ tsenor::ScoreSrc abs_source(const float* scores, int64_t ld) {
 int make_source(const tsenor_scores_t* d, int64_t cols, tsenor::ScoreSrc* out) {
     if (!d) return TSENOR_ERR_NULL;
     if (d->kind < TSENOR_SCORES_ABS || d->kind > TSENOR_SCORES_COLMUL) return TSENOR_ERR_ARG;
-    if (d->w_is_bf16 && d->kind != TSENOR_SCORES_COLMUL) return TSENOR_ERR_ARG;
     if (d->ld < cols) return TSENOR_ERR_SHAPE;
     if (!d->w) return TSENOR_ERR_NULL;
     tsenor::ScoreSrc S{};

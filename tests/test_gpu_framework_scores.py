@@ -36,6 +36,8 @@ def _sources(rows, cols, seed):
         ("coldiv", ts.Scores(ts.SCORES_COLDIV, Wd, colvec=dd), oracle.scores(oracle.SCORES_COLDIV, W, colvec=d)),
         ("colmul", ts.Scores(ts.SCORES_COLMUL, Wd, colvec=ad), oracle.scores(oracle.SCORES_COLMUL, W, colvec=a)),
         ("colmul_bf16", ts.Scores(ts.SCORES_COLMUL, Wb.to(DEV), colvec=ad), oracle.scores(oracle.SCORES_COLMUL, Wb32, colvec=a)),
+        ("abs_bf16", ts.Scores(ts.SCORES_ABS, Wb.to(DEV)), oracle.scores(oracle.SCORES_ABS, Wb32)),
+        ("admm_bf16", ts.Scores(ts.SCORES_ADMM, Wb.to(DEV), v=Vd, scalar=0.5), oracle.scores(oracle.SCORES_ADMM, Wb32, V, np.float32(0.5))),
     ]
 
 
@@ -127,7 +129,8 @@ def test_descriptor_errors():
     with pytest.raises(ts.TsenorError) as e:
         ts.scores_max(bad)
     assert e.value.status == ts.ERR_NULL
-    bf = ts.Scores(ts.SCORES_ABS, W.to(torch.bfloat16))             # bf16 only with COLMUL
+    src = ts.Scores(ts.SCORES_ABS, W)
+    src.desc.kind = 7                                               # unknown kind
     with pytest.raises(ts.TsenorError) as e:
-        ts.scores_materialize(bf)
+        ts.scores_materialize(src)
     assert e.value.status == ts.ERR_ARG
