@@ -483,3 +483,28 @@ def test_simple_rounding_properties_and_ablation_order():
     o_greedy = oracle.objective(W, oracle.round_plan(x, W, N, M, ls_steps=0))
     o_full = oracle.objective(W, oracle.round_plan(x, W, N, M))
     assert o_simple < o_greedy <= o_full
+
+
+def test_log_domain_oracle_equals_algorithm1_in_its_printed_linear_form():
+    """Algorithm 1 as printed works on S and Q themselves (no logarithms).  Written out here
+    in numpy for a tau that keeps exp(tau w) inside fp64, it must give the oracle's exp(x) and
+    exp(q) at every iteration count, cap active or not."""
+    rng = np.random.default_rng(41)
+    for M, N, tau in [(4, 2, 8.0), (8, 4, 25.0), (16, 8, 40.0), (8, 3, 25.0), (32, 16, 60.0)]:
+        w = np.abs(rng.standard_normal((M, M)))
+        w /= w.max()
+        S = np.exp(tau * w)
+        Q = np.ones((M, M))
+        done = 0
+        for iters in (1, 2, 3, 10, 60):
+            for _ in range(iters - done):
+                S = S * (N / S.sum(1, keepdims=True))          # line 3: Diag(N / (S 1)) S
+                S = S * (N / S.sum(0, keepdims=True))          # line 4: S Diag(N / (S^T 1))
+                Snew = np.minimum(S * Q, 1.0)                  # line 5
+                Q = Q * (S / Snew)                             # line 6
+                S = Snew
+            done = iters
+            x, q = oracle.dykstra_block(w, N, tau, iters)
+            assert np.allclose(np.exp(x), S, rtol=1e-9, atol=1e-300)
+            assert np.allclose(np.exp(q), Q, rtol=1e-9)
+        assert (S == 1.0).any()                                # the cap was active on the way
