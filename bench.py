@@ -140,7 +140,7 @@ def aggregate_rate(units_per_rank_per_step, steps, world, elapsed_ms):
     return world * units_per_rank_per_step * steps / (elapsed_ms / 1e3)
 
 
-WORKLOADS = ("config4", "config0", "config1", "config2", "config3", "config5", "admm", "wanda")
+WORKLOADS = ("config4", "config0", "config1", "config2", "config3", "config5", "admm", "wanda", "sparsegpt")
 
 
 class Job:
@@ -180,6 +180,12 @@ def make_jobs(workload, index):
         a = rng.lognormal(0.0, 1.0, size=4096).astype(np.float32)
         j = Job("wanda-8:16", 8, 16, {"w": W.view(torch.int16).numpy(), "a": a}, kind="wanda")
         return [j]
+    if workload == "sparsegpt":   # eight consecutive column groups (14336 x 32 slabs) of one matrix
+        W = (rng.standard_normal((14336, 256), dtype=np.float32) * np.float32(0.02))
+        d = (np.abs(rng.standard_normal(256)) + 0.05).astype(np.float32)
+        return [Job(f"group{g}-16:32", 16, 32, {"w": np.ascontiguousarray(W[:, 32 * g:32 * g + 32]),
+                                                "d": np.ascontiguousarray(d[32 * g:32 * g + 32])}, kind="coldiv")
+                for g in range(8)]
     raise ValueError(workload)
 
 
@@ -195,6 +201,8 @@ WORKLOAD_TEXT = {
     "admm": "ADMM D-update on 14336x4096: scores (W+V/rho)^2 computed in the loader, 16:32, then the "
             "keep-previous-mask safeguard",
     "wanda": "Wanda scores |W_ij| a_j computed in the loader from bf16 W (4096x4096) and fp32 a_j, 8:16",
+    "sparsegpt": "SparseGPT column groups: eight 14336x32 slabs solved one after the other (latency case: 448 "
+                 "blocks per call), scores |W_ij / d_j| computed in the loader, 16:32",
 }
 
 
@@ -225,6 +233,8 @@ def oracle_sample(job, blocks_wanted):
         import torch
         wf = torch.from_numpy(w).view(torch.bfloat16).to(torch.float32).numpy()
         full = oracle.scores(oracle.SCORES_COLMUL, wf, colvec=job.arrays["a"])
+    elif job.kind == "coldiv":
+        full = oracle.scores(oracle.SCORES_COLDIV, w, colvec=job.arrays["d"])
     else:
         full = w
     return np.ascontiguousarray(full[: nrows * M]), nrows * per_row, float(full.max())
@@ -316,6 +326,8 @@ def run_cuda(args, rank, world, local_rank):
                 return ts.Scores(ts.SCORES_ADMM, t["w"], v=t["v"], scalar=j.scalar)
             if j.kind == "wanda":
                 return ts.Scores(ts.SCORES_COLMUL, t["w"].view(torch.bfloat16), colvec=t["a"])
+            if j.kind == "coldiv":
+                return ts.Scores(ts.SCORES_COLDIV, t["w"], colvec=t["d"])
             return ts.Scores(ts.SCORES_ABS, t["w"])
 
         def solve(self, tensors, src, stream=None):

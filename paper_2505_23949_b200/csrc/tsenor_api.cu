@@ -73,12 +73,16 @@ int make_source(const tsenor_scores_t* d, int64_t cols, tsenor::ScoreSrc* out) {
 template <int M, int MODE>
 int launch(const tsenor::Params& P, cudaStream_t st) {
     using G = tsenor::Geom<M>;
+    // a slab (single block column) is cut into panels of vertically stacked blocks
+    const bool tall = (P.cols == M) && (P.rows > M);
+    constexpr int NB = G::PANEL / M;
     const int64_t npc = (P.cols + G::PANEL - 1) / G::PANEL;
-    const int64_t panels = (P.rows / M) * npc;
+    const int64_t panels = tall ? (P.rows / M + NB - 1) / NB : (P.rows / M) * npc;
     if (panels == 0) return TSENOR_OK;
     if (panels > 0x7fffffffLL) return TSENOR_ERR_SHAPE;
     tsenor::Params Q = P;
     Q.npc = (int)npc;
+    Q.tall = tall ? 1 : 0;
     const size_t smem = sizeof(tsenor::SmemLayout<M, MODE>);
     static thread_local int configured_device = -1;
     int dev = 0;

@@ -425,21 +425,37 @@ __device__ __forceinline__ int any_nonfinite(const float4& v) {
 }
 
 // ---------------------------------------------------------------------------
+// Where a panel's cells live in the matrix.  Wide matrices: the panel is M rows
+// x PANEL columns at (r0, c0).  Slabs (a single block column, cols == M, as in
+// the column groups of SparseGPT): the panel's blocks are stacked vertically,
+// block b of the panel being rows [(first + b) M, (first + b + 1) M), so that a
+// CTA still gets a full set of blocks and the whole slab is one wave of CTAs.
+// In shared memory both look the same: block b occupies columns [b M, b M + M).
+// ---------------------------------------------------------------------------
+template <int M> struct PanelMap {
+    int tall;
+    int64_t r0, c0;        // wide: origin of the panel
+    int64_t first;         // tall: first block (= block row) of the panel
+    int valid_cols;        // columns of the shared-memory panel that hold blocks
+    __device__ __forceinline__ int64_t row(int r, int c) const { return tall ? (first + c / M) * M + r : r0 + r; }
+    __device__ __forceinline__ int64_t col(int c) const { return tall ? (int64_t)(c % M) : c0 + c; }
+};
+
+// ---------------------------------------------------------------------------
 // Panel loaders: an M x PANEL panel into shared memory, coalesced, vector
 // loads when the addresses allow it.  Return non-zero if a non-finite value
 // was seen by this thread.
 // ---------------------------------------------------------------------------
 template <int M>
-__device__ __forceinline__ int load_score_panel(const ScoreSrc& S, int64_t r0, int64_t c0, int64_t cols,
+__device__ __forceinline__ int load_score_panel(const ScoreSrc& S, const PanelMap<M>& pm,
                                                 float* __restrict__ dst) {
     using G = Geom<M>;
     constexpr int V = G::PANEL / 4;
     int bad = 0;
     for (int idx = threadIdx.x; idx < M * V; idx += WARPS * 32) {
         const int r = idx / V, c = (idx % V) * 4;
-        const int64_t gc = c0 + c;
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (gc < cols) v = load_score_quad(S, r0 + r, gc);  // cols % 4 == 0: a quad is all in or all out
+        if (c < pm.valid_cols) v = load_score_quad(S, pm.row(r, c), pm.col(c));  // a quad is all in or all out
         bad |= any_nonfinite(v);
         float* d = dst + r * G::WS + c;
         d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
@@ -448,17 +464,16 @@ __device__ __forceinline__ int load_score_panel(const ScoreSrc& S, int64_t r0, i
 }
 
 template <int M>
-__device__ __forceinline__ int load_key_panel(const float* __restrict__ src, int64_t ld, int64_t r0, int64_t c0,
-                                              int64_t cols, bool vec_ok, float* __restrict__ dst) {
+__device__ __forceinline__ int load_key_panel(const float* __restrict__ src, int64_t ld, const PanelMap<M>& pm,
+                                              bool vec_ok, float* __restrict__ dst) {
     using G = Geom<M>;
     constexpr int V = G::PANEL / 4;
     int bad = 0;
     for (int idx = threadIdx.x; idx < M * V; idx += WARPS * 32) {
         const int r = idx / V, c = (idx % V) * 4;
-        const int64_t gc = c0 + c;
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (gc < cols) {
-            const float* p = src + (r0 + r) * ld + gc;
+        if (c < pm.valid_cols) {
+            const float* p = src + pm.row(r, c) * ld + pm.col(c);
             if (vec_ok) v = __ldg(reinterpret_cast<const float4*>(p));
             else v = make_float4(__ldg(p), __ldg(p + 1), __ldg(p + 2), __ldg(p + 3));
         }
@@ -715,6 +730,7 @@ struct Params {
     uint32_t* bits;      int64_t wpr;
     int64_t rows, cols;
     int npc;                       // panels per block row
+    int tall;                      // slab: one block column, panels stacked vertically
     int N; float Nf, log2N;
     float c_hi, c_lo;              // tau * log2(e), split in two floats
     int iters, ls_steps;
@@ -749,15 +765,26 @@ __global__ void __launch_bounds__(WARPS * 32, MinBlocks<M>::value) tsenor_kernel
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t panel = blockIdx.x;
-    const int64_t r0 = (panel / P.npc) * M;
-    const int64_t c0 = (panel % P.npc) * (int64_t)G::PANEL;
-    const int valid_cols = (int)((P.cols - c0 < G::PANEL) ? (P.cols - c0) : G::PANEL);
+    PanelMap<M> pm;
+    pm.tall = P.tall;
+    if (P.tall) {
+        constexpr int NB = G::PANEL / M;
+        const int64_t left = P.rows / M - panel * NB;
+        pm.first = panel * NB; pm.r0 = 0; pm.c0 = 0;
+        pm.valid_cols = (int)(left < NB ? left : NB) * M;
+    } else {
+        pm.r0 = (panel / P.npc) * M;
+        pm.c0 = (panel % P.npc) * (int64_t)G::PANEL;
+        pm.first = 0;
+        pm.valid_cols = (int)((P.cols - pm.c0 < G::PANEL) ? (P.cols - pm.c0) : G::PANEL);
+    }
+    const int valid_cols = pm.valid_cols;
     int flags = 0;
 
     // ---- block loader
-    if (load_score_panel<M>(P.src, r0, c0, P.cols, sm.w)) flags |= DEV_NONFINITE;
+    if (load_score_panel<M>(P.src, pm, sm.w)) flags |= DEV_NONFINITE;
     if (MODE == 2)
-        if (load_key_panel<M>(P.keys, P.ld_keys, r0, c0, P.cols, P.vec_keys != 0, sm.k)) flags |= DEV_NONFINITE;
+        if (load_key_panel<M>(P.keys, P.ld_keys, pm, P.vec_keys != 0, sm.k)) flags |= DEV_NONFINITE;
     if (MODE != 1)
         for (int idx = threadIdx.x; idx < M * G::WORDS; idx += WARPS * 32) sm.bits[idx] = 0u;
     __syncthreads();
@@ -809,8 +836,8 @@ __global__ void __launch_bounds__(WARPS * 32, MinBlocks<M>::value) tsenor_kernel
                 for (int a = 0; a < MR; ++a)
 #pragma unroll
                     for (int b = 0; b < MC; ++b) {
-                        const int64_t row = r0 + lr * MR + (a ^ gr);
-                        const int64_t col = c0 + blk * M + lc * MC + (b ^ gc);
+                        const int pc = blk * M + lc * MC + (b ^ gc);
+                        const int64_t row = pm.row(lr * MR + (a ^ gr), pc), col = pm.col(pc);
                         P.plan[row * P.ld_plan + col] = P.plan_is_log ? t[a][b] * 0.6931471805599453f : exp2f(t[a][b]);
                     }
             }
@@ -843,10 +870,18 @@ __global__ void __launch_bounds__(WARPS * 32, MinBlocks<M>::value) tsenor_kernel
             __syncwarp();
         }
         __syncthreads();
-        const int nwords = (valid_cols + 31) / 32;
-        for (int idx = threadIdx.x; idx < M * G::WORDS; idx += WARPS * 32) {
-            const int r = idx / G::WORDS, wd = idx % G::WORDS;
-            if (wd < nwords) P.bits[(r0 + r) * P.wpr + c0 / 32 + wd] = sm.bits[idx];
+        if (P.tall) {   // one word (M bits) per matrix row
+            constexpr unsigned GM = (M == 32) ? 0xffffffffu : ((1u << (M & 31)) - 1u);
+            for (int idx = threadIdx.x; idx < valid_cols; idx += WARPS * 32) {
+                const int blk = idx / M, r = idx % M;
+                P.bits[((pm.first + blk) * M + r) * P.wpr] = (sm.bits[r * G::WORDS + (blk * M) / 32] >> ((blk * M) % 32)) & GM;
+            }
+        } else {
+            const int nwords = (valid_cols + 31) / 32;
+            for (int idx = threadIdx.x; idx < M * G::WORDS; idx += WARPS * 32) {
+                const int r = idx / G::WORDS, wd = idx % G::WORDS;
+                if (wd < nwords) P.bits[(pm.r0 + r) * P.wpr + pm.c0 / 32 + wd] = sm.bits[idx];
+            }
         }
     }
     flags = __reduce_or_sync(FULL, flags);

@@ -77,6 +77,37 @@ def test_unaligned_and_strided_sources():
     assert oracle.count_infeasible(m, 32, 264, 4, 8) == 0
 
 
+@pytest.mark.parametrize("M,N", [(4, 2), (8, 4), (16, 8), (32, 16)])
+def test_sparsegpt_column_groups(M, N):
+    """SparseGPT walks a weight matrix in groups of M columns and prunes each rows x M slab with
+    the score |W_ij / d_j|: every group is a strided view into the wide matrix."""
+    rng = np.random.default_rng(100 + M)
+    rows, cols = M * 37, M * 5
+    W = (rng.standard_normal((rows, cols)) * 0.02).astype(np.float32)
+    d = (np.abs(rng.standard_normal(cols)) + 0.05).astype(np.float32)
+    Wd, dd = _dev(W), _dev(d)
+    full = np.zeros((rows, (cols + 31) // 32), np.uint32)
+    for g in range(cols // M):
+        c0 = g * M
+        src = ts.Scores(ts.SCORES_COLDIV, Wd[:, c0:c0 + M], colvec=dd[c0:c0 + M].contiguous())
+        ref = oracle.scores(oracle.SCORES_COLDIV, W[:, c0:c0 + M], colvec=d[c0:c0 + M])
+        assert np.array_equal(ts.scores_materialize(src).cpu().numpy(), ref)
+        tau = float(200.0 / ts.scores_max(src).item())
+        st = ts.new_status(DEV)
+        m = _bits(ts.solve_scores(src, N, M, tau, 300, status=st))
+        assert int(st.item()) == 0 and m.shape == (rows, 1)
+        assert oracle.count_infeasible(m, rows, M, N, M) == 0
+        want = oracle.solve(ref, N, M, tau, 300)
+        assert abs(oracle.objective(ref, m) - oracle.objective(ref, want)) <= 1e-4 * oracle.objective(ref, want)
+        # the slab path and the wide path of the same kernel agree block for block
+        wide = np.ascontiguousarray(ref.reshape(rows // M, M, M).transpose(1, 0, 2).reshape(M, rows))
+        mw = oracle.unpack_mask(_bits(ts.solve(_dev(wide), N, M, tau, 300)), rows)
+        assert np.array_equal(mw.reshape(M, rows // M, M).transpose(1, 0, 2).reshape(rows, M),
+                              oracle.unpack_mask(m, M))
+        full[:, c0 // 32] |= m[:, 0] << np.uint32(c0 % 32)
+    assert oracle.count_infeasible(full, rows, cols, N, M) == 0
+
+
 def test_admm_sequence_with_safeguard_matches_oracle():
     """A short ADMM-like sequence: the score matrix drifts, every iteration solves and keeps
     the previous mask if the new one retains less (Appendix A.1.3)."""

@@ -27,6 +27,12 @@ SHAPES = [
     (32, 7, 64, 160),
     (4, 1, 8, 516),
     (4, 3, 8, 516),
+    # slabs (one block column, as the column groups of SparseGPT): several stacked panels + a tail
+    (4, 2, 4 * 259, 4),
+    (8, 4, 8 * 131, 8),
+    (16, 8, 16 * 35, 16),
+    (32, 16, 32 * 11, 32),
+    (32, 16, 32, 32),
 ]
 
 
