@@ -49,6 +49,10 @@ def lib():
         L.oracle_solve.argtypes = [_f32p, i64, i64, i64, i32, i32, f32, i32, i32,
                                    _u32p, vp, vp, vp, C.POINTER(i64)]
         L.oracle_solve.restype = i32
+        L.oracle_dykstra_blocktau.argtypes = L.oracle_dykstra.argtypes
+        L.oracle_dykstra_blocktau.restype = i32
+        L.oracle_solve_blocktau.argtypes = L.oracle_solve.argtypes
+        L.oracle_solve_blocktau.restype = i32
         L.oracle_objective.argtypes = [_f32p, i64, _u32p, i64, i64]
         L.oracle_objective.restype = f64
         L.oracle_count_infeasible.argtypes = [_u32p, i64, i64, i32, i32]
@@ -151,12 +155,14 @@ def mask_words_per_row(cols):
     return (int(cols) + 31) // 32
 
 
-def dykstra(scores, N, M, tau, iters, plan_is_log=False):
-    """Algorithm 1 on every aligned M x M tile; fp64 plan in matrix layout."""
+def dykstra(scores, N, M, tau, iters, plan_is_log=False, per_block_tau=False):
+    """Algorithm 1 on every aligned M x M tile; fp64 plan in matrix layout.  With
+    ``per_block_tau`` every block runs with tau / (its own largest score)."""
     s = _f32(scores)
     rows, cols = s.shape
     plan = np.empty((rows, cols), np.float64)
-    _check(lib().oracle_dykstra(s, rows, cols, cols, int(N), int(M), float(tau),
+    fn = lib().oracle_dykstra_blocktau if per_block_tau else lib().oracle_dykstra
+    _check(fn(s, rows, cols, cols, int(N), int(M), float(tau),
                                 int(iters), plan, cols, int(bool(plan_is_log))), "dykstra")
     return plan
 
@@ -189,16 +195,18 @@ def round_plan(plan_key, scores, N, M, ls_steps=-1, stats=False):
     return bits
 
 
-def solve(scores, N, M, tau, iters, ls_steps=-1, stats=False):
+def solve(scores, N, M, tau, iters, ls_steps=-1, stats=False, per_block_tau=False):
     """Algorithm 1 (fp64) + Algorithm 2 on every tile.  Returns the packed
-    mask, or ``(mask, info)`` with per-block statistics."""
+    mask, or ``(mask, info)`` with per-block statistics.  With ``per_block_tau``
+    every block runs with tau / (its own largest score)."""
     s = _f32(scores)
     rows, cols = s.shape
     bits = np.zeros((rows, mask_words_per_row(cols)), np.uint32)
     nblk = (rows // M) * (cols // M)
     st, npz, ob, ptrs = _stats_arrays(nblk, stats)
     bad = C.c_int64(0)
-    _check(lib().oracle_solve(s, rows, cols, cols, int(N), int(M), float(tau),
+    fn = lib().oracle_solve_blocktau if per_block_tau else lib().oracle_solve
+    _check(fn(s, rows, cols, cols, int(N), int(M), float(tau),
                               int(iters), int(ls_steps), bits, *ptrs, C.byref(bad)), "solve")
     if stats:
         return bits, dict(steps=st, nonpos=npz, obj=ob, underfilled=bad.value)

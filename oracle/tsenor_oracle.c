@@ -344,8 +344,20 @@ static void gather_block_abs(const float *scores, int64_t ld, int64_t r0,
  * plan_out (rows x cols doubles, leading dimension ld_plan) gets S = exp(x),
  * or x = log S when plan_is_log is non-zero, in matrix layout.
  */
-int oracle_dykstra(const float *scores, int64_t rows, int64_t cols, int64_t ld,
-                   int N, int M, float tau, int iters, double *plan_out,
+/* tau of one block: the caller's tau, or (per-block variant) tau_rel divided by
+ * the block's own largest score, i.e. the parameter rule of Appendix B.1 applied
+ * block by block instead of to the whole matrix. */
+static double tau_of_block(double tau, int per_block, const double *w, int M)
+{
+    if (!per_block) return tau;
+    double m = 0.0;
+    for (int e = 0; e < M * M; ++e)
+        if (w[e] > m) m = w[e];
+    return m > 0.0 ? tau / m : 0.0;
+}
+
+static int dykstra_matrix(const float *scores, int64_t rows, int64_t cols, int64_t ld,
+                   int N, int M, float tau, int per_block, int iters, double *plan_out,
                    int64_t ld_plan, int plan_is_log)
 {
     if (!scores || !plan_out || !check_shape(rows, cols, N, M) || iters < 0 ||
@@ -360,7 +372,7 @@ int oracle_dykstra(const float *scores, int64_t rows, int64_t cols, int64_t ld,
         for (int64_t b = 0; b < nbr * nbc; ++b) {
             int64_t r0 = (b / nbc) * M, c0 = (b % nbc) * M;
             gather_block_abs(scores, ld, r0, c0, M, w, NULL);
-            oracle_dykstra_block(w, M, N, (double)tau, iters, 0, x, q);
+            oracle_dykstra_block(w, M, N, tau_of_block((double)tau, per_block, w, M), iters, 0, x, q);
             for (int i = 0; i < M; ++i)
                 for (int j = 0; j < M; ++j)
                     plan_out[(size_t)(r0 + i) * ld_plan + (c0 + j)] =
@@ -461,8 +473,8 @@ int oracle_round(const float *plan_key, int64_t ld_plan, const float *scores,
  * fp64 sort key of Algorithm 2, local search on the fp32 scores.  Outputs as
  * in oracle_round.
  */
-int oracle_solve(const float *scores, int64_t rows, int64_t cols, int64_t ld,
-                 int N, int M, float tau, int iters, int ls_steps,
+static int solve_matrix(const float *scores, int64_t rows, int64_t cols, int64_t ld,
+                 int N, int M, float tau, int per_block, int iters, int ls_steps,
                  uint32_t *mask_bits, int32_t *blk_steps, int32_t *blk_nonpos,
                  double *blk_obj, int64_t *underfilled)
 {
@@ -484,7 +496,7 @@ int oracle_solve(const float *scores, int64_t rows, int64_t cols, int64_t ld,
             for (int64_t bc = 0; bc < nbc; ++bc) {
                 int64_t r0 = br * M, c0 = bc * M, b = br * nbc + bc;
                 gather_block_abs(scores, ld, r0, c0, M, w, wf);
-                oracle_dykstra_block(w, M, N, (double)tau, iters, 0, x, q);
+                oracle_dykstra_block(w, M, N, tau_of_block((double)tau, per_block, w, M), iters, 0, x, q);
                 int steps, nonpos;
                 double obj;
                 int ok = round_one(x, wf, M, N, ls_steps, S, R, C, &steps,
@@ -502,6 +514,39 @@ int oracle_solve(const float *scores, int64_t rows, int64_t cols, int64_t ld,
     }
     if (underfilled) *underfilled = bad;
     return ORACLE_OK;
+}
+
+int oracle_solve(const float *scores, int64_t rows, int64_t cols, int64_t ld,
+                 int N, int M, float tau, int iters, int ls_steps,
+                 uint32_t *mask_bits, int32_t *blk_steps, int32_t *blk_nonpos,
+                 double *blk_obj, int64_t *underfilled)
+{
+    return solve_matrix(scores, rows, cols, ld, N, M, tau, 0, iters, ls_steps, mask_bits,
+                        blk_steps, blk_nonpos, blk_obj, underfilled);
+}
+
+/* Per-block variant: block b runs with tau = tau_rel / max|score| of block b. */
+int oracle_solve_blocktau(const float *scores, int64_t rows, int64_t cols, int64_t ld,
+                          int N, int M, float tau_rel, int iters, int ls_steps,
+                          uint32_t *mask_bits, int32_t *blk_steps, int32_t *blk_nonpos,
+                          double *blk_obj, int64_t *underfilled)
+{
+    return solve_matrix(scores, rows, cols, ld, N, M, tau_rel, 1, iters, ls_steps, mask_bits,
+                        blk_steps, blk_nonpos, blk_obj, underfilled);
+}
+
+int oracle_dykstra(const float *scores, int64_t rows, int64_t cols, int64_t ld,
+                   int N, int M, float tau, int iters, double *plan_out,
+                   int64_t ld_plan, int plan_is_log)
+{
+    return dykstra_matrix(scores, rows, cols, ld, N, M, tau, 0, iters, plan_out, ld_plan, plan_is_log);
+}
+
+int oracle_dykstra_blocktau(const float *scores, int64_t rows, int64_t cols, int64_t ld,
+                            int N, int M, float tau_rel, int iters, double *plan_out,
+                            int64_t ld_plan, int plan_is_log)
+{
+    return dykstra_matrix(scores, rows, cols, ld, N, M, tau_rel, 1, iters, plan_out, ld_plan, plan_is_log);
 }
 
 /* Objective of Eq. 1: sum of |score| over the set bits, in fp64. */

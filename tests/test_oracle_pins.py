@@ -508,3 +508,28 @@ def test_log_domain_oracle_equals_algorithm1_in_its_printed_linear_form():
             assert np.allclose(np.exp(x), S, rtol=1e-9, atol=1e-300)
             assert np.allclose(np.exp(q), Q, rtol=1e-9)
         assert (S == 1.0).any()                                # the cap was active on the way
+
+
+def test_per_block_tau_is_the_plain_method_block_by_block():
+    """The per-block variant must equal running the method on each block alone with
+    tau = tau_rel / max of that block, and must help when one column dwarfs the rest."""
+    M, N, nb = 8, 4, 5
+    W = np.abs(np.random.default_rng(51).standard_normal((M * nb, M * nb)) * 0.02).astype(np.float32)
+    W[:, 3] *= 20
+    bits = oracle.solve(W, N, M, 200.0, 300, per_block_tau=True)
+    plan = oracle.dykstra(W, N, M, 200.0, 40, per_block_tau=True)
+    dense = oracle.unpack_mask(bits, M * nb)
+    for b in range(nb * nb):
+        r0, c0 = (b // nb) * M, (b % nb) * M
+        blk = np.ascontiguousarray(W[r0:r0 + M, c0:c0 + M])
+        one = oracle.unpack_mask(oracle.solve(blk, N, M, 200.0 / blk.max(), 300), M)
+        assert np.array_equal(dense[r0:r0 + M, c0:c0 + M], one)
+        # (the stand-alone call rounds its tau to fp32, the per-block one divides in fp64)
+        assert np.allclose(plan[r0:r0 + M, c0:c0 + M], oracle.dykstra(blk, N, M, 200.0 / blk.max(), 40), rtol=1e-4)
+    opt = sum(_lp_optimum(W[(b // nb) * M:(b // nb + 1) * M, (b % nb) * M:(b % nb + 1) * M].astype(np.float64), N)
+              for b in range(nb * nb))
+    gap_pb = opt - oracle.objective(W, bits)
+    gap_gl = opt - oracle.objective(W, oracle.solve(W, N, M, 200.0 / W.max(), 300))
+    assert 0 <= gap_pb <= gap_gl
+    zero = np.zeros((M, M), np.float32)                    # an all-zero block gets tau = 0
+    assert oracle.count_infeasible(oracle.solve(zero, N, M, 200.0, 10, per_block_tau=True), M, M, N, M) == 0
