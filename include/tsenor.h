@@ -160,6 +160,10 @@ typedef struct tsenor_scores {
     int64_t ld_v;
     float scalar;        /* TSENOR_SCORES_ADMM: 1/rho                                  */
     const float *colvec; /* COLDIV / COLMUL: cols floats                               */
+    int per_block_tau;   /* non-zero: every block runs with tau / (largest score of that
+                            block) instead of tau, i.e. the parameter rule of
+                            Appendix B.1 applied block by block (pass tau = 200 for
+                            "entropy weight 0.005 max|W|"); an all-zero block gets 0  */
 } tsenor_scores_t;
 
 /* tsenor_solve on the score matrix described by *s (same arguments otherwise). */
@@ -167,6 +171,12 @@ int tsenor_solve_scores(const tsenor_scores_t *s, int64_t rows, int64_t cols,
                         int N, int M, float tau, int iters, int ls_steps,
                         uint32_t *mask_bits_out, int32_t *dev_status,
                         tsenor_stream_t stream);
+
+/* tsenor_dykstra on the score matrix described by *s (same arguments otherwise). */
+int tsenor_dykstra_scores(const tsenor_scores_t *s, int64_t rows, int64_t cols,
+                          int N, int M, float tau, int iters, float *plan_out,
+                          int64_t ld_plan, int plan_is_log, int32_t *dev_status,
+                          tsenor_stream_t stream);
 
 /* *dev_max_out = largest score of the described matrix (for the choice of tau). */
 int tsenor_scores_max(const tsenor_scores_t *s, int64_t rows, int64_t cols,

@@ -21,7 +21,7 @@ EXPORTS = (
     "tsenor_solve", "tsenor_dykstra", "tsenor_round", "tsenor_objective", "tsenor_check",
     "tsenor_max_abs", "tsenor_mask_words_per_row", "tsenor_strerror", "tsenor_last_cuda_error",
     "tsenor_launch_count", "tsenor_solve_scores", "tsenor_scores_max", "tsenor_scores_materialize",
-    "tsenor_keep_better", "tsenor_simple_round",
+    "tsenor_keep_better", "tsenor_simple_round", "tsenor_dykstra_scores",
 )
 
 SCORES_ABS, SCORES_ADMM, SCORES_COLDIV, SCORES_COLMUL = 0, 1, 2, 3
@@ -30,7 +30,8 @@ SCORES_ABS, SCORES_ADMM, SCORES_COLDIV, SCORES_COLMUL = 0, 1, 2, 3
 class ScoresDesc(C.Structure):
     """ctypes image of ``tsenor_scores_t`` (a host struct holding device pointers)."""
     _fields_ = [("kind", C.c_int), ("w_is_bf16", C.c_int), ("w", C.c_void_p), ("ld", C.c_int64),
-                ("v", C.c_void_p), ("ld_v", C.c_int64), ("scalar", C.c_float), ("colvec", C.c_void_p)]
+                ("v", C.c_void_p), ("ld_v", C.c_int64), ("scalar", C.c_float), ("colvec", C.c_void_p),
+                ("per_block_tau", C.c_int)]
 
 _lib = None
 
@@ -65,6 +66,8 @@ def lib():
             getattr(L, name).restype = i32
         sp = C.POINTER(ScoresDesc)
         L.tsenor_solve_scores.argtypes = [sp, i64, i64, i32, i32, f32, i32, i32, vp, vp, vp]
+        L.tsenor_dykstra_scores.argtypes = [sp, i64, i64, i32, i32, f32, i32, vp, i64, i32, vp, vp]
+        L.tsenor_dykstra_scores.restype = i32
         L.tsenor_scores_max.argtypes = [sp, i64, i64, vp, vp]
         L.tsenor_scores_materialize.argtypes = [sp, i64, i64, vp, i64, vp]
         L.tsenor_keep_better.argtypes = [sp, i64, i64, vp, vp, vp, vp]
@@ -193,7 +196,7 @@ class Scores:
     the descriptor.  kind: SCORES_ABS |W|, SCORES_ADMM (W + V*scalar)^2, SCORES_COLDIV
     |W / colvec_j|, SCORES_COLMUL |W| * colvec_j.  W may be float32 or bfloat16."""
 
-    def __init__(self, kind, w, v=None, scalar=0.0, colvec=None):
+    def __init__(self, kind, w, v=None, scalar=0.0, colvec=None, per_block_tau=False):
         if not (isinstance(w, torch.Tensor) and w.is_cuda and w.dim() == 2 and w.stride(1) == 1):
             raise TypeError("w must be a 2-D row-major CUDA tensor")
         if w.dtype not in (torch.float32, torch.bfloat16):
@@ -216,6 +219,7 @@ class Scores:
                     and colvec.numel() == self.cols):
                 raise TypeError("colvec must be a contiguous float32 CUDA vector of length cols")
             d.colvec = colvec.data_ptr()
+        d.per_block_tau = int(bool(per_block_tau))
         self.desc = d
 
     @property
@@ -232,6 +236,18 @@ def solve_scores(src, N, M, tau, iters=300, ls_steps=-1, mask_out=None, status=N
     if rc:
         raise TsenorError(rc, "tsenor_solve_scores")
     return mask_out
+
+
+def dykstra_scores(src, N, M, tau, iters=300, plan_is_log=False, plan_out=None, status=None, stream=None):
+    """tsenor_dykstra_scores: Algorithm 1 only on a described score matrix."""
+    if plan_out is None:
+        plan_out = torch.empty((src.rows, src.cols), dtype=torch.float32, device=src.device)
+    pp, _, _, ldp = _mat(plan_out, "plan_out")
+    rc = lib().tsenor_dykstra_scores(C.byref(src.desc), src.rows, src.cols, int(N), int(M), float(tau), int(iters),
+                                     pp, ldp, int(bool(plan_is_log)), _ptr(status), _stream(stream))
+    if rc:
+        raise TsenorError(rc, "tsenor_dykstra_scores")
+    return plan_out
 
 
 def scores_max(src, out=None, stream=None):

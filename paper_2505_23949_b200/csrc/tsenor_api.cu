@@ -310,8 +310,9 @@ int trivial_mask(uint32_t* bits, int64_t rows, int64_t cols, bool ones, cudaStre
 
 extern "C" {
 
-static int solve_on(const tsenor::ScoreSrc& src, int64_t rows, int64_t cols, int N, int M, float tau, int iters,
-                    int ls_steps, uint32_t* mask_bits_out, int32_t* dev_status, cudaStream_t st) {
+static int solve_on(const tsenor::ScoreSrc& src, int per_block_tau, int64_t rows, int64_t cols, int N, int M,
+                    float tau, int iters, int ls_steps, uint32_t* mask_bits_out, int32_t* dev_status,
+                    cudaStream_t st) {
     if (N == 0 || N == M) return trivial_mask(mask_bits_out, rows, cols, N == M, st);
     tsenor::Params P{};
     P.src = src;
@@ -319,6 +320,7 @@ static int solve_on(const tsenor::ScoreSrc& src, int64_t rows, int64_t cols, int
     P.rows = rows; P.cols = cols;
     P.N = N; P.Nf = (float)N; P.log2N = (float)std::log2((double)N);
     set_tau(P, tau);
+    P.per_block_tau = per_block_tau;
     P.iters = iters; P.ls_steps = ls_steps;
     P.status = dev_status;
     return dispatch<0>(P, M, st);
@@ -331,7 +333,7 @@ int tsenor_solve(const float* scores, int64_t rows, int64_t cols, int64_t ld, in
     if (iters < 0 || !(tau >= 0.0f) || !std::isfinite(tau)) return TSENOR_ERR_ARG;
     if (rows == 0 || cols == 0) return TSENOR_OK;
     if (!scores || !mask_bits_out) return TSENOR_ERR_NULL;
-    return solve_on(abs_source(scores, ld), rows, cols, N, M, tau, iters, ls_steps, mask_bits_out, dev_status,
+    return solve_on(abs_source(scores, ld), 0, rows, cols, N, M, tau, iters, ls_steps, mask_bits_out, dev_status,
                     (cudaStream_t)stream);
 }
 
@@ -344,7 +346,8 @@ int tsenor_solve_scores(const tsenor_scores_t* s, int64_t rows, int64_t cols, in
     if (int rc = make_source(s, cols, &src)) return rc;
     if (rows == 0 || cols == 0) return TSENOR_OK;
     if (!mask_bits_out) return TSENOR_ERR_NULL;
-    return solve_on(src, rows, cols, N, M, tau, iters, ls_steps, mask_bits_out, dev_status, (cudaStream_t)stream);
+    return solve_on(src, s->per_block_tau ? 1 : 0, rows, cols, N, M, tau, iters, ls_steps, mask_bits_out, dev_status,
+                    (cudaStream_t)stream);
 }
 
 static int max_on(const tsenor::ScoreSrc& src, int64_t rows, int64_t cols, float* dev_max_out, cudaStream_t st) {
@@ -409,6 +412,21 @@ int tsenor_simple_round(const float* plan_key, int64_t ld_plan, int64_t rows, in
     return finish_launch();
 }
 
+static int dykstra_on(const tsenor::ScoreSrc& src, int per_block_tau, int64_t rows, int64_t cols, int N, int M,
+                      float tau, int iters, float* plan_out, int64_t ld_plan, int plan_is_log,
+                      int32_t* dev_status, cudaStream_t st) {
+    tsenor::Params P{};
+    P.src = src;
+    P.plan = plan_out; P.ld_plan = ld_plan; P.plan_is_log = plan_is_log;
+    P.rows = rows; P.cols = cols;
+    P.N = N; P.Nf = (float)N; P.log2N = (float)std::log2((double)N);
+    set_tau(P, tau);
+    P.per_block_tau = per_block_tau;
+    P.iters = iters; P.ls_steps = -1;
+    P.status = dev_status;
+    return dispatch<1>(P, M, st);
+}
+
 int tsenor_dykstra(const float* scores, int64_t rows, int64_t cols, int64_t ld, int N, int M, float tau, int iters,
                    float* plan_out, int64_t ld_plan, int plan_is_log, int32_t* dev_status, tsenor_stream_t stream) {
     if (!valid_M(M) || N < 1 || N >= M) return TSENOR_ERR_NM;
@@ -417,15 +435,23 @@ int tsenor_dykstra(const float* scores, int64_t rows, int64_t cols, int64_t ld, 
     if (iters < 0 || !(tau >= 0.0f) || !std::isfinite(tau)) return TSENOR_ERR_ARG;
     if (rows == 0 || cols == 0) return TSENOR_OK;
     if (!scores || !plan_out) return TSENOR_ERR_NULL;
-    tsenor::Params P{};
-    P.src = abs_source(scores, ld);
-    P.plan = plan_out; P.ld_plan = ld_plan; P.plan_is_log = plan_is_log;
-    P.rows = rows; P.cols = cols;
-    P.N = N; P.Nf = (float)N; P.log2N = (float)std::log2((double)N);
-    set_tau(P, tau);
-    P.iters = iters; P.ls_steps = -1;
-    P.status = dev_status;
-    return dispatch<1>(P, M, (cudaStream_t)stream);
+    return dykstra_on(abs_source(scores, ld), 0, rows, cols, N, M, tau, iters, plan_out, ld_plan, plan_is_log,
+                      dev_status, (cudaStream_t)stream);
+}
+
+int tsenor_dykstra_scores(const tsenor_scores_t* s, int64_t rows, int64_t cols, int N, int M, float tau, int iters,
+                          float* plan_out, int64_t ld_plan, int plan_is_log, int32_t* dev_status,
+                          tsenor_stream_t stream) {
+    if (!valid_M(M) || N < 1 || N >= M) return TSENOR_ERR_NM;
+    if (int rc = check_matrix(rows, cols, cols, M)) return rc;
+    if (ld_plan < cols) return TSENOR_ERR_SHAPE;
+    if (iters < 0 || !(tau >= 0.0f) || !std::isfinite(tau)) return TSENOR_ERR_ARG;
+    tsenor::ScoreSrc src{};
+    if (int rc = make_source(s, cols, &src)) return rc;
+    if (rows == 0 || cols == 0) return TSENOR_OK;
+    if (!plan_out) return TSENOR_ERR_NULL;
+    return dykstra_on(src, s->per_block_tau ? 1 : 0, rows, cols, N, M, tau, iters, plan_out, ld_plan, plan_is_log,
+                      dev_status, (cudaStream_t)stream);
 }
 
 int tsenor_round(const float* plan_key, int64_t ld_plan, const float* scores, int64_t ld, int64_t rows,

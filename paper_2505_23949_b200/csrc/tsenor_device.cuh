@@ -733,6 +733,7 @@ struct Params {
     int tall;                      // slab: one block column, panels stacked vertically
     int N; float Nf, log2N;
     float c_hi, c_lo;              // tau * log2(e), split in two floats
+    int per_block_tau;             // tau is divided by each block's own largest score
     int iters, ls_steps;
     int32_t* status;
     int vec_keys;
@@ -810,14 +811,30 @@ __global__ void __launch_bounds__(WARPS * 32, MinBlocks<M>::value) tsenor_kernel
             }
             mx[a] = m;
         }
-        if (P.iters > 0) {
+        float c_hi = P.c_hi, c_lo = P.c_lo;
+        if (P.iters > 0 || P.per_block_tau) {
             reduce_scatter<MR, PC>(mx, 1, OpMax());
             all_gather<MR, PC>(mx, 1);
+        }
+        if (P.per_block_tau) {   // tau of this block = tau_rel / its largest score
+            float bm = mx[0];
+#pragma unroll
+            for (int a = 1; a < MR; ++a) bm = fmaxf(bm, mx[a]);
+#pragma unroll
+            for (int s = 0; (1 << s) < PR; ++s) bm = fmaxf(bm, __shfl_xor_sync(FULL, bm, PC << s));
+            if (bm > 0.0f) {
+                c_hi = __fdiv_rn(P.c_hi, bm);
+                c_lo = __fdiv_rn(fmaf(-c_hi, bm, P.c_hi) + P.c_lo, bm);
+            } else {
+                c_hi = 0.0f; c_lo = 0.0f;
+            }
+        }
+        if (P.iters > 0) {
 #pragma unroll
             for (int a = 0; a < MR; ++a) {
-                const float sh = mx[a] * P.c_hi;
+                const float sh = mx[a] * c_hi;
 #pragma unroll
-                for (int b = 0; b < MC; ++b) t[a][b] = fmaf(t[a][b], P.c_lo, fmaf(t[a][b], P.c_hi, -sh));
+                for (int b = 0; b < MC; ++b) t[a][b] = fmaf(t[a][b], c_lo, fmaf(t[a][b], c_hi, -sh));
             }
             dykstra_iterate<M>(t, sm.k + warp * (32 * MR * MC), lane, P.Nf, P.log2N, P.iters);
 #pragma unroll
@@ -828,7 +845,7 @@ __global__ void __launch_bounds__(WARPS * 32, MinBlocks<M>::value) tsenor_kernel
 #pragma unroll
             for (int a = 0; a < MR; ++a)
 #pragma unroll
-                for (int b = 0; b < MC; ++b) t[a][b] = fmaf(t[a][b], P.c_lo, t[a][b] * P.c_hi);
+                for (int b = 0; b < MC; ++b) t[a][b] = fmaf(t[a][b], c_lo, t[a][b] * c_hi);
         }
         if (MODE == 1) {
             if (active) {

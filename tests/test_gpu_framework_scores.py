@@ -165,3 +165,26 @@ def test_descriptor_errors():
     with pytest.raises(ts.TsenorError) as e:
         ts.scores_materialize(src)
     assert e.value.status == ts.ERR_ARG
+
+
+@pytest.mark.parametrize("M,N,rows,cols", [(32, 16, 64, 352), (16, 8, 32, 592), (8, 4, 24, 1096), (4, 2, 16, 1060)])
+def test_per_block_tau_matches_oracle(M, N, rows, cols):
+    """tau divided by each block's own largest score (Appendix B.1 rule applied per block)."""
+    W = synth.gaussian_outlier_columns_abs(rows, cols, 0.02, 77 + M, frac=0.01)
+    W[0:M, 0:M] = 0.0                                               # an all-zero block: tau = 0 there
+    src = ts.Scores(ts.SCORES_ABS, _dev(W), per_block_tau=True)
+    st = ts.new_status(DEV)
+    plan = ts.dykstra_scores(src, N, M, 200.0, 300, status=st).cpu().numpy()
+    ref = oracle.dykstra(W, N, M, 200.0, 300, per_block_tau=True)
+    assert np.abs(plan - ref).max() <= 1e-4
+    mask = _bits(ts.solve_scores(src, N, M, 200.0, 300, status=st))
+    assert int(st.item()) == 0
+    assert oracle.count_infeasible(mask, rows, cols, N, M) == 0
+    want = oracle.solve(W, N, M, 200.0, 300, per_block_tau=True)
+    o_gpu, o_ref = oracle.objective(W, mask), oracle.objective(W, want)
+    assert abs(o_gpu - o_ref) <= 1e-4 * o_ref
+    # and it retains more than the whole-matrix rule when a few columns dominate
+    glob = _bits(ts.solve(_dev(W), N, M, synth.default_tau(W.max()), 300))
+    assert o_gpu >= oracle.objective(W, glob)
+    # iters = 0 uses the same per-block scaling (key = tau_b |w|: same order as |w| inside a block)
+    assert np.array_equal(_bits(ts.solve_scores(src, N, M, 200.0, 0)), oracle.round_plan(W, W, N, M))
