@@ -147,7 +147,7 @@ struct Comp {
 // (one multiply per element less, three shuffles more): pays off except at M = 32.
 template <int M> struct LazyRow { static constexpr bool value = (M != 32); };
 constexpr int CHECK = 4;     // iterations between range tests of the accumulated scalings
-constexpr int MAXRUN = 24;   // longest run of linear-domain iterations (multiple of CHECK)
+constexpr int MAXRUN = 48;   // longest run of linear-domain iterations (multiple of CHECK)
 
 template <int M>
 __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>::MC], float* stash, int lane,
