@@ -1,0 +1,84 @@
+"""Randomised GPU-vs-oracle cases: shapes, N:M, tau, iteration counts, repair modes, key
+distributions and leading dimensions drawn from a seeded generator."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2505_23949_b200 import binding as ts
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _bits(t):
+    return t.cpu().numpy().view(np.uint32)
+
+
+def _case(rng):
+    M = int(rng.choice([4, 8, 16, 32]))
+    N = int(rng.integers(1, M))
+    rows = M * int(rng.integers(1, 6))
+    cols = M * int(rng.integers(1, 40)) if rng.random() < 0.85 else M
+    kind = rng.integers(0, 4)
+    if kind == 0:
+        W = np.abs(rng.standard_normal((rows, cols)))
+    elif kind == 1:
+        W = np.abs(rng.standard_t(2.5, (rows, cols)))
+    elif kind == 2:
+        W = np.round(np.abs(rng.standard_normal((rows, cols))) * 4) / 4      # many equal scores
+    else:
+        W = np.abs(rng.standard_normal((rows, cols))) * np.where(rng.random(cols) < 0.05, 30.0, 1.0)[None, :]
+    W = (W * 10.0 ** rng.uniform(-3, 1)).astype(np.float32)
+    return M, N, rows, cols, W
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_rounding_cases_are_bit_exact(seed):
+    rng = np.random.default_rng(9000 + seed)
+    for _ in range(25):
+        M, N, rows, cols, W = _case(rng)
+        mode = rng.integers(0, 3)
+        if mode == 0:
+            key = rng.standard_normal((rows, cols)).astype(np.float32)
+        elif mode == 1:
+            key = np.minimum(rng.standard_normal((rows, cols)) * 3, 0).astype(np.float32)
+        else:
+            key = (np.round(rng.standard_normal((rows, cols)) * 2) / 2).astype(np.float32)
+        ls = int(rng.choice([-1, -1, 0, 1, 3, 10]))
+        pad = int(rng.integers(0, 3))
+        kd = torch.zeros((rows, cols + pad), device=DEV)[:, :cols]
+        kd.copy_(torch.from_numpy(key))
+        wd = torch.zeros((rows, cols + 2 * pad), device=DEV)[:, pad:pad + cols]
+        wd.copy_(torch.from_numpy(W))
+        st = ts.new_status(DEV)
+        got = _bits(ts.round_plan(kd, wd, N, M, ls_steps=ls, status=st))
+        want, info = oracle.round_plan(key, W, N, M, ls_steps=ls, stats=True)
+        assert np.array_equal(got, want), (seed, M, N, rows, cols, ls)
+        assert (int(st.item()) & ts.DEV_INTERNAL) == 0
+        assert bool(int(st.item()) & ts.DEV_UNDERFILLED) == (info["underfilled"] > 0)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_solve_cases_match_the_oracle(seed):
+    rng = np.random.default_rng(7000 + seed)
+    for _ in range(12):
+        M, N, rows, cols, W = _case(rng)
+        tau = float(rng.choice([20.0, 60.0, 200.0]) / W.max())
+        iters = int(rng.choice([1, 2, 5, 30, 100, 300]))
+        Wd = torch.from_numpy(W).to(DEV)
+        st = ts.new_status(DEV)
+        plan = ts.dykstra(Wd, N, M, tau, iters, status=st).cpu().numpy()
+        ref = oracle.dykstra(W, N, M, tau, iters)
+        assert np.abs(plan - ref).max() <= 1e-4, (seed, M, N, rows, cols, iters)
+        got = _bits(ts.solve(Wd, N, M, tau, iters, status=st))
+        assert int(st.item()) == 0
+        assert oracle.count_infeasible(got, rows, cols, N, M) == 0
+        if iters >= 100:
+            # After a handful of iterations hundreds of plan entries sit within rounding of the cap,
+            # the greedy order among them is decided by noise (exact ties in fp64, 1e-7 apart in
+            # fp32) and masks legitimately differ; the objective is compared once the plan has
+            # separated, as at the method's operating point T = 300.
+            want = oracle.solve(W, N, M, tau, iters)
+            o_gpu, o_ref = oracle.objective(W, got), oracle.objective(W, want)
+            assert abs(o_gpu - o_ref) <= 2e-3 * o_ref, (seed, M, N, rows, cols, iters)
