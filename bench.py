@@ -39,10 +39,11 @@ NCU_DRAM_BYTES_PER_LAUNCH = 250.91e6   # 235.04 MB read + 15.87 MB written
 
 def fp32_lane_ops_per_block(M, T):
     """fp32 lane operations one block needs in the kernel's formulation of Algorithm 1: per
-    element and iteration the clip (min), one row-sum add, one column-sum fma and the two
-    scalings by rho_i and kappa_j.  Reductions across lanes, reciprocals, the occasional exp2
-    rebuild of the iterate and the rounding stage are overhead, not counted."""
-    return 5 * M * M * T
+    element and iteration the clip (a min against the moving threshold 1/R_i), one row-sum
+    add, one column-sum fma and the scaling by kappa_j (the row scaling is folded into the
+    threshold).  Reductions across lanes, reciprocals, the occasional exp2 rebuild of the
+    iterate and the rounding stage are overhead, not counted."""
+    return 4 * M * M * T
 
 
 def xu_ops_per_block_one_exp(M, T):
@@ -465,10 +466,13 @@ def run_cuda(args, rank, world, local_rank):
                     "d2h_bytes_per_step": sum(d.mask.numel() * 4 for d in djobs)},
             "gpu_launches": launches,
             "roofline": {
-                "bound": "alu", "pipe": "fp32 dispatch (add/mul/fma/min), 5 lane-ops per element and iteration",
+                "bound": "alu", "pipe": "fp32 dispatch (add/mul/fma/min), 4 lane-ops per element and iteration",
                 "achieved": achieved / 1e12, "peak": fp32_peak / 1e12, "unit": "Tlaneop/s",
                 "frac": achieved / fp32_peak,
-                "frac_fma_pipe_only": achieved * 0.8 / fp32_peak,
+                # time a kernel doing the scope table's per-unit fp32 work (9 M^2 T, its one-exp model;
+                # 12 M^2 T for the paper's listing) would need at that peak, over the measured time
+                "vs_fp32_bound_one_exp_model": achieved * 9 / 4 / fp32_peak,
+                "vs_fp32_bound_paper_listing": achieved * 12 / 4 / fp32_peak,
                 "peak_source": f"148 SMs x 128 fp32 lanes/clk x sm_max_mhz ({peak_kind} clock)",
                 "kernel": "tsenor_kernel<M,0>" if len(jobs) > 2 else f"tsenor_kernel<{jobs[0].M},0>",
                 "launch_ms": 1e3 * solve_s / (args.steps * nj),

@@ -120,7 +120,8 @@ struct Comp {
 //     kap_j  = N / sum_i e_ij rho_i                (projection on C2)
 //     U_ij  <- U_ij rho_i kap_j ,  F_i += log2 rho_i ,  G_j += log2 kap_j
 // with the clip (C3) and the dual update implicit in the next e.  U is the
-// linear-domain iterate of Algorithm 1.  It is trusted only while the scalings
+// linear-domain iterate of Algorithm 1 (kept as U / R_i in the registers, see
+// the loop below).  It is trusted only while the scalings
 // applied since it was last rebuilt stay small, and is then rebuilt as
 // 2^(t0 + F + G) from the log-domain potentials; that is what keeps large
 // tau |w| safe in fp32.  Every CHECK iterations the products of rho_i and of
@@ -143,9 +144,6 @@ struct Comp {
 // holds the final t = x + q.  stash: 32 * MR * MC floats of shared memory
 // private to the warp (keeps t0 while the registers hold U).
 // ---------------------------------------------------------------------------
-// Whether the row scalings are folded into the clip threshold instead of the tile
-// (one multiply per element less, three shuffles more): pays off except at M = 32.
-template <int M> struct LazyRow { static constexpr bool value = (M != 32); };
 constexpr int CHECK = 4;     // iterations between range tests of the accumulated scalings
 constexpr int MAXRUN = 48;   // longest run of linear-domain iterations (multiple of CHECK)
 
@@ -211,8 +209,14 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>:
         }
     }
     // Iterations 1 .. iters-1.  Element-wise work runs on pairs of columns with
-    // the packed fp32x2 add / mul / fma of sm_100 (half the issue slots).
-    float2 U[MR][MP];
+    // the packed fp32x2 add / mul / fma of sm_100 (half the issue slots).  The row
+    // scalings are never applied to the tile: the registers hold V = U / R_i with
+    // R_i the product of the rho_i since the last rebuild, so that
+    // e = R_i min(V, 1/R_i): the clip threshold moves instead of the tile, the new
+    // R_i is simply N / sum_j min(V_ij, 1/R_i), the column sums are
+    // sum_i min(V_ij, 1/R_i) R_i(new), and one multiply per element (by kap_j) is
+    // left.  Four fp32 operations per element and iteration: min, add, fma, mul.
+    float2 V[MR][MP];
     float iR[MR];
     const float invN = 1.0f / Nf;
     int run = MAXRUN;                          // linear-domain iterations since the last rebuild
@@ -243,14 +247,11 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>:
                 const float2 x0 = __fadd2_rn(__fadd2_rn(make_float2(v.x, v.y), Fa), make_float2(G[2 * b], G[2 * b + 1]));
                 const float2 x1 =
                     __fadd2_rn(__fadd2_rn(make_float2(v.z, v.w), Fa), make_float2(G[2 * b + 2], G[2 * b + 3]));
-                U[a][b] = make_float2(ex2_approx(x0.x), ex2_approx(x0.y));
-                U[a][b + 1] = make_float2(ex2_approx(x1.x), ex2_approx(x1.y));
+                V[a][b] = make_float2(ex2_approx(x0.x), ex2_approx(x0.y));
+                V[a][b + 1] = make_float2(ex2_approx(x1.x), ex2_approx(x1.y));
             }
         }
         ++run;
-      if (LazyRow<M>::value) {
-        // Row scalings stay out of the tile: it holds V = U / R_i (R_i = product of the
-        // rho_i since the rebuild), e = R_i min(V, 1/R_i); the new R_i is N / sum_j min(..).
         if (rebuild) {
 #pragma unroll
             for (int a = 0; a < MR; ++a) iR[a] = 1.0f;
@@ -262,7 +263,7 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>:
             float2 s2;
 #pragma unroll
             for (int b = 0; b < MP; ++b) {
-                m[a][b] = make_float2(fminf(U[a][b].x, iR[a]), fminf(U[a][b].y, iR[a]));
+                m[a][b] = make_float2(fminf(V[a][b].x, iR[a]), fminf(V[a][b].y, iR[a]));
                 s2 = (b == 0) ? m[a][b] : __fadd2_rn(s2, m[a][b]);
             }
             rp[a] = s2.x + s2.y;
@@ -295,51 +296,8 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>:
         for (int a = 0; a < MR; ++a) {
             iR[a] = iRn[a];
 #pragma unroll
-            for (int b = 0; b < MP; ++b) U[a][b] = __fmul2_rn(U[a][b], make_float2(kap[2 * b], kap[2 * b + 1]));
+            for (int b = 0; b < MP; ++b) V[a][b] = __fmul2_rn(V[a][b], make_float2(kap[2 * b], kap[2 * b + 1]));
         }
-      } else {
-        float2 e[MR][MP];
-        float rp[MR], rho[MR], cp[MC], kap[MC];
-#pragma unroll
-        for (int a = 0; a < MR; ++a) {
-            float2 s2;
-#pragma unroll
-            for (int b = 0; b < MP; ++b) {
-                e[a][b] = make_float2(fminf(U[a][b].x, 1.0f), fminf(U[a][b].y, 1.0f));
-                s2 = (b == 0) ? e[a][b] : __fadd2_rn(s2, e[a][b]);
-            }
-            rp[a] = s2.x + s2.y;
-        }
-        reduce_scatter<MR, PC>(rp, 1, OpAdd());
-#pragma unroll
-        for (int k = 0; k < RO; ++k) {
-            rho[k] = Nf * rcp_approx(rp[k]);
-            Pr[k] *= rho[k];
-        }
-        all_gather<MR, PC>(rho, 1);
-#pragma unroll
-        for (int b = 0; b < MP; ++b) {
-            float2 c2 = __fmul2_rn(e[0][b], make_float2(rho[0], rho[0]));
-#pragma unroll
-            for (int a = 1; a < MR; ++a) c2 = __ffma2_rn(e[a][b], make_float2(rho[a], rho[a]), c2);
-            cp[2 * b] = c2.x;
-            cp[2 * b + 1] = c2.y;
-        }
-        reduce_scatter<MC, PR>(cp, PC, OpAdd());
-#pragma unroll
-        for (int k = 0; k < CO; ++k) {
-            kap[k] = Nf * rcp_approx(cp[k]);
-            Pc[k] *= kap[k];
-        }
-        all_gather<MC, PR>(kap, PC);
-#pragma unroll
-        for (int a = 0; a < MR; ++a) {
-            const float2 ra = make_float2(rho[a], rho[a]);
-#pragma unroll
-            for (int b = 0; b < MP; ++b)
-                U[a][b] = __fmul2_rn(__fmul2_rn(U[a][b], ra), make_float2(kap[2 * b], kap[2 * b + 1]));
-        }
-      }
     }
     // final potentials and t = t0 + F + G
 #pragma unroll
