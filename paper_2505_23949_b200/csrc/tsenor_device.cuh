@@ -712,7 +712,7 @@ template <int M> struct SmemLayout<M, 1> {   // Algorithm 1 alone: score panel a
     unsigned int bits[1];
 };
 // Resident CTAs per SM the register allocation aims for.
-template <int M> struct MinBlocks { static constexpr int value = (M == 32) ? 6 : ((M == 4) ? 5 : 4); };
+template <int M> struct MinBlocks { static constexpr int value = (M == 4) ? 5 : 4; };
 
 template <int M, int MODE>
 __global__ void __launch_bounds__(WARPS * 32, MinBlocks<M>::value) tsenor_kernel(const Params P) {
