@@ -100,8 +100,8 @@ def test_dykstra_literal_small_tau_and_tau_zero():
 def test_rounding_is_bit_exact(keykind, M, N, rows, cols):
     rng = np.random.default_rng(1000 * M + N)
     W = _scores("wanda" if keykind == "ties" else "gauss", rows, cols, 31 * M + N)
-    if keykind == "plan":      # the log-plan the GPU itself produced (fp32)
-        key = ts.dykstra(_dev(W), N, M, synth.default_tau(W.max()), 300, plan_is_log=True).cpu().numpy()
+    if keykind == "plan":      # the oracle's log-plan, rounded to fp32: the same array for both sides
+        key = oracle.dykstra(W, N, M, synth.default_tau(W.max()), 300, plan_is_log=True).astype(np.float32)
     elif keykind == "ties":    # few distinct values: the index tie-break decides almost everything
         key = np.round(rng.standard_normal((rows, cols)) * 1.5).astype(np.float32)
         key[::3, ::5] = -0.0
