@@ -36,20 +36,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
-def build_ubench() -> str:
-    """Compiles the fp32-dispatch micro-benchmark (evidence for the roofline, not part of the
-    library) into ``build/ubench_fp32_dispatch`` at the repository root."""
-    out_dir = os.path.join(ROOT, "build")
-    os.makedirs(out_dir, exist_ok=True)
-    exe = os.path.join(out_dir, "ubench_fp32_dispatch")
-    subprocess.run(["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-o", exe,
-                    os.path.join(CSRC, "ubench_fp32_dispatch.cu")], check=True)
-    return exe
-
-
 if __name__ == "__main__":
     import sys
-    if "--ubench" in sys.argv:
-        print(build_ubench())
-    else:
-        print(build(force=True, verbose="-v" in sys.argv))
+    print(build(force=True, verbose="-v" in sys.argv))

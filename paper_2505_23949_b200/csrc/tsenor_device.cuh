@@ -147,6 +147,81 @@ struct Comp {
 constexpr int CHECK = 4;     // iterations between range tests of the accumulated scalings
 constexpr int MAXRUN = 48;   // longest run of linear-domain iterations (multiple of CHECK)
 
+__device__ __forceinline__ bool out_of_window(float p) {
+    const unsigned e = (__float_as_uint(p) >> 23) & 0xffu;
+    return (e - 111u) > 32u && e != 255u;
+}
+
+// One iteration t >= 1 on the linear-domain iterate.  Element-wise work runs on
+// pairs of columns with the packed fp32x2 add / mul / fma of sm_100 (half the
+// issue slots).  The row scalings are never applied to the tile: the registers
+// hold V = U / R_i with R_i the product of the rho_i since the last rebuild, and
+// one multiply per element (by kap_j) is left.  Four fp32 operations per element
+// and iteration, in one of two forms:
+//   SAT  (M >= 16)  rs[a] = R_i:    e = sat(V R_i) = min(U, 1) by a saturating multiply
+//                   (FMA pipe), row sums of e give rho_i = N / sum, column sums are
+//                   sum_i e_ij rho_i, R_i <- R_i rho_i in every lane of the row;
+//   !SAT (M <= 8)   rs[a] = 1/R_i:  m = min(V, 1/R_i) (the clip threshold moves
+//                   instead of the tile), the new R_i is simply N / sum_j m_ij and
+//                   the column sums are sum_i m_ij R_i(new).
+// Both compute the same iterate; which one is faster depends on how the ALU pipe
+// (fp32 min) and the FMA pipe are loaded at that block size (measured).
+template <int M> struct UseSat { static constexpr bool value = (M >= 16); };
+
+template <int M>
+__device__ __forceinline__ void dykstra_step(float2 (&V)[Tile<M>::MR][Tile<M>::MC / 2], float (&rs)[Tile<M>::MR],
+                                             float (&Pr)[Tile<M>::MR / Tile<M>::PC],
+                                             float (&Pc)[Tile<M>::MC / Tile<M>::PR], float Nf, float invN) {
+    using T = Tile<M>;
+    constexpr int MR = T::MR, MC = T::MC, PR = T::PR, PC = T::PC;
+    constexpr int RO = MR / PC, CO = MC / PR, MP = MC / 2;
+    constexpr bool SAT = UseSat<M>::value;
+    float2 m[MR][MP];
+    float rp[MR], sc[MR], thr[MR], cp[MC], kap[MC];
+#pragma unroll
+    for (int a = 0; a < MR; ++a) {
+        float2 s2;
+#pragma unroll
+        for (int b = 0; b < MP; ++b) {
+            if (SAT) m[a][b] = make_float2(__saturatef(V[a][b].x * rs[a]), __saturatef(V[a][b].y * rs[a]));
+            else m[a][b] = make_float2(fminf(V[a][b].x, rs[a]), fminf(V[a][b].y, rs[a]));
+            s2 = (b == 0) ? m[a][b] : __fadd2_rn(s2, m[a][b]);
+        }
+        rp[a] = s2.x + s2.y;
+    }
+    reduce_scatter<MR, PC>(rp, 1, OpAdd());
+#pragma unroll
+    for (int k = 0; k < RO; ++k) {
+        sc[k] = Nf * rcp_approx(rp[k]);          // SAT: rho_i; !SAT: the new R_i
+        if (SAT) Pr[k] *= sc[k];
+        else { Pr[k] = sc[k]; thr[k] = rp[k] * invN; }
+    }
+    all_gather<MR, PC>(sc, 1);
+    if (!SAT) all_gather<MR, PC>(thr, 1);
+#pragma unroll
+    for (int b = 0; b < MP; ++b) {
+        float2 c2 = __fmul2_rn(m[0][b], make_float2(sc[0], sc[0]));
+#pragma unroll
+        for (int a = 1; a < MR; ++a) c2 = __ffma2_rn(m[a][b], make_float2(sc[a], sc[a]), c2);
+        cp[2 * b] = c2.x;
+        cp[2 * b + 1] = c2.y;
+    }
+    reduce_scatter<MC, PR>(cp, PC, OpAdd());
+#pragma unroll
+    for (int k = 0; k < CO; ++k) {
+        kap[k] = Nf * rcp_approx(cp[k]);
+        Pc[k] *= kap[k];
+    }
+    all_gather<MC, PR>(kap, PC);
+#pragma unroll
+    for (int a = 0; a < MR; ++a) {
+        if (SAT) rs[a] *= sc[a];
+        else rs[a] = thr[a];
+#pragma unroll
+        for (int b = 0; b < MP; ++b) V[a][b] = __fmul2_rn(V[a][b], make_float2(kap[2 * b], kap[2 * b + 1]));
+    }
+}
+
 template <int M>
 __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>::MC], float* stash, int lane,
                                                 float Nf, float log2N, int iters) {
@@ -156,7 +231,7 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>:
     constexpr int MP = MC / 2, NQ = MR * MC / 4;
     float F[MR], G[MC];
     Comp Fo[RO], Go[CO];
-    float Pr[RO], Pc[CO];                      // products of rho / kap since the last resync
+    float Pr[RO], Pc[CO];                      // products of rho / kap since the last rebuild
     if (iters <= 0) return;
     float4* const st4 = reinterpret_cast<float4*>(stash) + lane;
 #pragma unroll
@@ -208,96 +283,53 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>:
             Pc[k] = 1.0f;
         }
     }
-    // Iterations 1 .. iters-1.  Element-wise work runs on pairs of columns with
-    // the packed fp32x2 add / mul / fma of sm_100 (half the issue slots).  The row
-    // scalings are never applied to the tile: the registers hold V = U / R_i with
-    // R_i the product of the rho_i since the last rebuild, so that
-    // e = R_i min(V, 1/R_i): the clip threshold moves instead of the tile, the new
-    // R_i is simply N / sum_j min(V_ij, 1/R_i), the column sums are
-    // sum_i min(V_ij, 1/R_i) R_i(new), and one multiply per element (by kap_j) is
-    // left.  Four fp32 operations per element and iteration: min, add, fma, mul.
+    // Iterations 1 .. iters-1 in runs: rebuild U from the potentials, then groups of
+    // CHECK iterations with the range test of the accumulated scalings between groups.
     float2 V[MR][MP];
-    float iR[MR];
+    float rs[MR];
     const float invN = 1.0f / Nf;
-    int run = MAXRUN;                          // linear-domain iterations since the last rebuild
-#pragma unroll(M >= 16 ? 4 : 1)   // several iterations per trip help the large tiles by 1-2 %
-    for (int it = 1; it < iters; ++it) {
-        bool rebuild = (run >= MAXRUN);
-        if (!rebuild && (run % CHECK) == 0) {
-            // exponent field in [127-16, 127+16] <=> product in [2^-16, 2^17)
-            bool wide = false;
+    int it = 1;
+#pragma unroll 1
+    while (it < iters) {
 #pragma unroll
-            for (int k = 0; k < RO; ++k) wide |= (((__float_as_uint(Pr[k]) >> 23) & 0xffu) - 111u) > 32u;
+        for (int k = 0; k < RO; ++k) { Fo[k].add(lg2_approx(Pr[k])); Pr[k] = 1.0f; F[k] = Fo[k].hi; }
 #pragma unroll
-            for (int k = 0; k < CO; ++k) wide |= (((__float_as_uint(Pc[k]) >> 23) & 0xffu) - 111u) > 32u;
-            rebuild = __any_sync(FULL, wide);
+        for (int k = 0; k < CO; ++k) { Go[k].add(lg2_approx(Pc[k])); Pc[k] = 1.0f; G[k] = Go[k].hi; }
+        all_gather<MR, PC>(F, 1);
+        all_gather<MC, PR>(G, PC);
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) {
+            const int a = (4 * q) / MC, b = ((4 * q) % MC) / 2;
+            const float4 v = st4[q * 32];
+            const float2 Fa = make_float2(F[a], F[a]);
+            const float2 x0 = __fadd2_rn(__fadd2_rn(make_float2(v.x, v.y), Fa), make_float2(G[2 * b], G[2 * b + 1]));
+            const float2 x1 =
+                __fadd2_rn(__fadd2_rn(make_float2(v.z, v.w), Fa), make_float2(G[2 * b + 2], G[2 * b + 3]));
+            V[a][b] = make_float2(ex2_approx(x0.x), ex2_approx(x0.y));
+            V[a][b + 1] = make_float2(ex2_approx(x1.x), ex2_approx(x1.y));
         }
-        if (rebuild) {
-            run = 0;
 #pragma unroll
-            for (int k = 0; k < RO; ++k) { Fo[k].add(lg2_approx(Pr[k])); Pr[k] = 1.0f; F[k] = Fo[k].hi; }
+        for (int a = 0; a < MR; ++a) rs[a] = 1.0f;     // R_i = 1 (and 1/R_i = 1)
+        const int run_end = (iters - it > MAXRUN) ? it + MAXRUN : iters;
+        bool wide = false;
+#pragma unroll 1
+        while (!wide && it + CHECK <= run_end) {
 #pragma unroll
-            for (int k = 0; k < CO; ++k) { Go[k].add(lg2_approx(Pc[k])); Pc[k] = 1.0f; G[k] = Go[k].hi; }
-            all_gather<MR, PC>(F, 1);
-            all_gather<MC, PR>(G, PC);
+            for (int u = 0; u < CHECK; ++u) dykstra_step<M>(V, rs, Pr, Pc, Nf, invN);
+            it += CHECK;
+            // exponent field in [127-16, 127+16] <=> product in [2^-16, 2^17).  A product that
+            // is inf or NaN (exponent field 255: a block poisoned by a non-finite score) does
+            // not vote, so that it cannot change when the other blocks of its warp rebuild.
+            bool w = false;
 #pragma unroll
-            for (int q = 0; q < NQ; ++q) {
-                const int a = (4 * q) / MC, b = ((4 * q) % MC) / 2;
-                const float4 v = st4[q * 32];
-                const float2 Fa = make_float2(F[a], F[a]);
-                const float2 x0 = __fadd2_rn(__fadd2_rn(make_float2(v.x, v.y), Fa), make_float2(G[2 * b], G[2 * b + 1]));
-                const float2 x1 =
-                    __fadd2_rn(__fadd2_rn(make_float2(v.z, v.w), Fa), make_float2(G[2 * b + 2], G[2 * b + 3]));
-                V[a][b] = make_float2(ex2_approx(x0.x), ex2_approx(x0.y));
-                V[a][b + 1] = make_float2(ex2_approx(x1.x), ex2_approx(x1.y));
-            }
+            for (int k = 0; k < RO; ++k) w |= out_of_window(Pr[k]);
+#pragma unroll
+            for (int k = 0; k < CO; ++k) w |= out_of_window(Pc[k]);
+            wide = __any_sync(FULL, w);
         }
-        ++run;
-        if (rebuild) {
-#pragma unroll
-            for (int a = 0; a < MR; ++a) iR[a] = 1.0f;
-        }
-        float2 m[MR][MP];
-        float rp[MR], Rn[MR], iRn[MR], cp[MC], kap[MC];
-#pragma unroll
-        for (int a = 0; a < MR; ++a) {
-            float2 s2;
-#pragma unroll
-            for (int b = 0; b < MP; ++b) {
-                m[a][b] = make_float2(fminf(V[a][b].x, iR[a]), fminf(V[a][b].y, iR[a]));
-                s2 = (b == 0) ? m[a][b] : __fadd2_rn(s2, m[a][b]);
-            }
-            rp[a] = s2.x + s2.y;
-        }
-        reduce_scatter<MR, PC>(rp, 1, OpAdd());
-#pragma unroll
-        for (int k = 0; k < RO; ++k) {
-            Pr[k] = Nf * rcp_approx(rp[k]);
-            Rn[k] = Pr[k];
-            iRn[k] = rp[k] * invN;
-        }
-        all_gather<MR, PC>(Rn, 1);
-        all_gather<MR, PC>(iRn, 1);
-#pragma unroll
-        for (int b = 0; b < MP; ++b) {
-            float2 c2 = __fmul2_rn(m[0][b], make_float2(Rn[0], Rn[0]));
-#pragma unroll
-            for (int a = 1; a < MR; ++a) c2 = __ffma2_rn(m[a][b], make_float2(Rn[a], Rn[a]), c2);
-            cp[2 * b] = c2.x;
-            cp[2 * b + 1] = c2.y;
-        }
-        reduce_scatter<MC, PR>(cp, PC, OpAdd());
-#pragma unroll
-        for (int k = 0; k < CO; ++k) {
-            kap[k] = Nf * rcp_approx(cp[k]);
-            Pc[k] *= kap[k];
-        }
-        all_gather<MC, PR>(kap, PC);
-#pragma unroll
-        for (int a = 0; a < MR; ++a) {
-            iR[a] = iRn[a];
-#pragma unroll
-            for (int b = 0; b < MP; ++b) V[a][b] = __fmul2_rn(V[a][b], make_float2(kap[2 * b], kap[2 * b + 1]));
+        if (!wide) {   // fewer than CHECK iterations left (end of the last run only)
+#pragma unroll 1
+            for (; it < run_end; ++it) dykstra_step<M>(V, rs, Pr, Pc, Nf, invN);
         }
     }
     // final potentials and t = t0 + F + G

@@ -485,18 +485,93 @@ def test_simple_rounding_properties_and_ablation_order():
     assert o_simple < o_greedy <= o_full
 
 
+def _simple_round_by_definition(k, N):
+    """Appendix B.2 "Simple", written out: keep the N best keys of every row, then the N best
+    of the survivors of every column; "best" = key descending, position ascending."""
+    M = k.shape[0]
+    S = np.zeros((M, M), np.uint8)
+    for i in range(M):
+        for j in sorted(range(M), key=lambda j: (-k[i, j], j))[:N]:
+            S[i, j] = 1
+    for j in range(M):
+        surv = [i for i in range(M) if S[i, j]]
+        for i in sorted(surv, key=lambda i: (-k[i, j], i))[N:]:
+            S[i, j] = 0
+    return S
+
+
+def test_simple_rounding_worked_examples_and_definition():
+    """Pins both passes of the "Simple" rounding.  Two blocks worked by hand (the dropped
+    entries are named), then the definition written out above on random, heavy-tie and
+    at-cap keys for every block size, N = M/2 and N != M/2."""
+    # 2:4, column 0 is the best entry of every row: rows keep {0, their second best}; column 0
+    # then has 4 survivors and keeps the two largest, 0.9 (row 2) and 0.8 (row 0): (1,0), (3,0) go.
+    k = np.array([[0.8, 0.1, 0.3, 0.2],
+                  [0.7, 0.2, 0.1, 0.6],
+                  [0.9, 0.5, 0.4, 0.3],
+                  [0.6, 0.1, 0.2, 0.5]], np.float32)
+    want = np.array([[1, 0, 1, 0],
+                     [0, 0, 0, 1],
+                     [1, 1, 0, 0],
+                     [0, 0, 0, 1]], np.uint8)
+    got = oracle.unpack_mask(oracle.simple_round(k, 2, 4), 4)
+    assert np.array_equal(got, want)
+    assert got[1, 0] == 0 and got[3, 0] == 0 and got[0, 0] == 1 and got[2, 0] == 1
+    # all keys equal (every comparison is a tie): rows keep columns 0 and 1, columns 0 and 1
+    # then keep rows 0 and 1 -- ties go to the smaller position in both passes
+    flat = oracle.unpack_mask(oracle.simple_round(np.zeros((4, 4), np.float32), 2, 4), 4)
+    assert np.array_equal(flat, np.array([[1, 1, 0, 0], [1, 1, 0, 0], [0, 0, 0, 0], [0, 0, 0, 0]], np.uint8))
+    # 1:4 with a tie inside a column: rows 0 and 2 both send their best entry to column 1 with
+    # the same key; the smaller row index survives
+    k1 = np.array([[0.1, 0.5, 0.2, 0.3],
+                   [0.9, 0.1, 0.2, 0.3],
+                   [0.2, 0.5, 0.1, 0.4],
+                   [0.1, 0.2, 0.3, 0.8]], np.float32)
+    got1 = oracle.unpack_mask(oracle.simple_round(k1, 1, 4), 4)
+    assert np.array_equal(got1, np.array([[0, 1, 0, 0], [1, 0, 0, 0], [0, 0, 0, 0], [0, 0, 0, 1]], np.uint8))
+
+    rng = np.random.default_rng(34)
+    seen_overfull = 0
+    for M, N in [(4, 2), (4, 1), (4, 3), (8, 4), (8, 3), (16, 8), (16, 5), (32, 16), (32, 7), (32, 25)]:
+        nb = 3
+        for kind in ("random", "ties", "cap"):
+            if kind == "random":
+                K = rng.standard_normal((M * nb, M * nb))
+            elif kind == "ties":
+                K = rng.integers(0, 4, (M * nb, M * nb)).astype(np.float64)
+            else:   # like a log-plan: many entries exactly at the cap (0), the rest negative
+                K = np.minimum(rng.standard_normal((M * nb, M * nb)) * 3 - 1, 0.0)
+            K = K.astype(np.float32)
+            dense = oracle.unpack_mask(oracle.simple_round(K, N, M), M * nb)
+            for b in range(nb * nb):
+                r0, c0 = (b // nb) * M, (b % nb) * M
+                k = K[r0:r0 + M, c0:c0 + M]
+                assert np.array_equal(dense[r0:r0 + M, c0:c0 + M], _simple_round_by_definition(k, N)), (M, N, kind)
+                rows_top = np.zeros((M, M), np.uint8)
+                for i in range(M):
+                    rows_top[i, sorted(range(M), key=lambda j: (-k[i, j], j))[:N]] = 1
+                seen_overfull += int((rows_top.sum(0) > N).any())
+    assert seen_overfull > 50          # the column pass had survivors to drop in most blocks
+
+
 def test_log_domain_oracle_equals_algorithm1_in_its_printed_linear_form():
     """Algorithm 1 as printed works on S and Q themselves (no logarithms).  Written out here
-    in numpy for a tau that keeps exp(tau w) inside fp64, it must give the oracle's exp(x) and
-    exp(q) at every iteration count, cap active or not."""
+    in numpy fp64 it must give the oracle's exp(x) and exp(q) at every iteration count, cap
+    active or not -- up to the operating point tau max(w) = 200 and T = 300, where exp(tau w)
+    reaches 7e86 (far outside fp32, which is why the method needs its log-domain form, but
+    inside fp64, so the printed form can still serve as the reference)."""
     rng = np.random.default_rng(41)
-    for M, N, tau in [(4, 2, 8.0), (8, 4, 25.0), (16, 8, 40.0), (8, 3, 25.0), (32, 16, 60.0)]:
+    cases = [(4, 2, 8.0, (1, 2, 3, 10, 60)), (8, 4, 25.0, (1, 2, 3, 10, 60)), (16, 8, 40.0, (1, 2, 3, 10, 60)),
+             (8, 3, 25.0, (1, 2, 3, 10, 60)), (32, 16, 60.0, (1, 2, 3, 10, 60)),
+             (4, 2, 200.0, (1, 5, 300)), (8, 4, 200.0, (1, 5, 300)), (16, 8, 200.0, (1, 5, 300)),
+             (32, 16, 200.0, (1, 2, 3, 10, 60, 300)), (32, 9, 200.0, (1, 300))]
+    for M, N, tau, counts in cases:
         w = np.abs(rng.standard_normal((M, M)))
         w /= w.max()
         S = np.exp(tau * w)
         Q = np.ones((M, M))
         done = 0
-        for iters in (1, 2, 3, 10, 60):
+        for iters in counts:
             for _ in range(iters - done):
                 S = S * (N / S.sum(1, keepdims=True))          # line 3: Diag(N / (S 1)) S
                 S = S * (N / S.sum(0, keepdims=True))          # line 4: S Diag(N / (S^T 1))
@@ -505,8 +580,10 @@ def test_log_domain_oracle_equals_algorithm1_in_its_printed_linear_form():
                 S = Snew
             done = iters
             x, q = oracle.dykstra_block(w, N, tau, iters)
-            assert np.allclose(np.exp(x), S, rtol=1e-9, atol=1e-300)
-            assert np.allclose(np.exp(q), Q, rtol=1e-9)
+            assert np.allclose(np.exp(x), S, rtol=1e-8, atol=1e-300), (M, N, tau, iters)
+            assert np.allclose(np.exp(q), Q, rtol=1e-8), (M, N, tau, iters)
+            if tau == 200.0:   # at the operating point also as an absolute bound on the plan
+                assert np.abs(np.exp(x) - S).max() < 1e-11
         assert (S == 1.0).any()                                # the cap was active on the way
 
 
