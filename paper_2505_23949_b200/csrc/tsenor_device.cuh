@@ -479,19 +479,18 @@ __device__ __forceinline__ int load_key_panel(const float* __restrict__ src, int
 // Rounding stage (Algorithm 2).  A group of M lanes owns one block; lane i of
 // the group plays row i and column i at once.
 // ---------------------------------------------------------------------------
-// Per-group scratch of the rounding stage.  The four byte tables that hold the
-// sorted orders (each lane only ever reads its own line of them) are written
-// over the block's own key cells once both sorts have consumed the keys: key
-// row i (M floats = 4M bytes) becomes
-//   [0,M)   rperm[p] -> column of the p-th best entry of row i
-//   [M,2M)  cperm[s] -> row of the s-th best entry of column i
-//   [2M,3M) rrank[j] -> rank of (i,j) inside row i
-//   [3M,4M) crank[r] -> rank of (r,i) inside column i
+// Tables of the rounding stage: for every line (row or column) of a block the
+// M prefix sets of its sorted order, prefix p = bit mask of the positions of its
+// p+1 best entries (uint32 words for M = 32, uint16 otherwise).  Each lane only
+// ever reads the two tables of its own row and column.  The row tables (and for
+// M <= 16 the column tables too) are written over the block's own key cells once
+// both sorts have consumed the keys: key row i (M floats = 4M bytes) becomes
+//   M = 32 :  [0,4M) row prefixes of row i          (column prefixes: SmemLayout::cpre)
+//   M <= 16:  [0,2M) row prefixes of row i, [2M,4M) column prefixes of column i
 template <int M> struct RoundScratch {
-    unsigned int rs[M];           // row-side picks of the round, bits over columns
-    unsigned int cs[M];           // column-side picks of the round, bits over rows
-    unsigned int sel[M];          // current mask, one word per row
+    unsigned int sel[M];          // current mask, one word per row (local search)
 };
+constexpr int CPRE_STRIDE = 33;   // words per column-prefix table at M = 32 (odd: conflict-free)
 
 // Strict order "key descending, index ascending" as one ascending u64.
 __device__ __forceinline__ unsigned long long sort_word(float key, int idx) {
@@ -536,124 +535,127 @@ template <int LO, int N, int M> __device__ __forceinline__ void oem_sort(unsigne
 }
 template <int M> __device__ __forceinline__ void sort_regs(unsigned long long (&v)[M]) { oem_sort<0, M, M>(v); }
 
-// Sorts one line (stride `st` floats in shared memory); returns the permutation
-// packed four indices per word (byte p%4 of word p/4 = index of the p-th best).
+// Sorts one line (stride `st` floats in shared memory) and returns the prefix sets of the
+// sorted order: pre[p] = positions of the p+1 best entries, packed two per word (16 bits
+// each) for M <= 16.
+template <int M> struct PreWords { static constexpr int value = (M == 32) ? 32 : M / 2; };
 template <int M>
-__device__ __forceinline__ void sort_line(const float* line, int st, unsigned (&packed)[M / 4]) {
+__device__ __forceinline__ void sort_line(const float* line, int st, unsigned (&pre)[PreWords<M>::value]) {
     unsigned long long v[M];
 #pragma unroll
     for (int k = 0; k < M; ++k) v[k] = sort_word(line[k * st], k);
     sort_regs<M>(v);
+    unsigned acc = 0u;
 #pragma unroll
-    for (int w = 0; w < M / 4; ++w)
-        packed[w] = ((unsigned)v[4 * w] & 63u) | (((unsigned)v[4 * w + 1] & 63u) << 8) |
-                    (((unsigned)v[4 * w + 2] & 63u) << 16) | (((unsigned)v[4 * w + 3] & 63u) << 24);
+    for (int p = 0; p < M; ++p) {
+        acc |= 1u << ((unsigned)v[p] & 31u);
+        if (M == 32) pre[p] = acc;
+        else if (p % 2 == 0) pre[p / 2] = acc;
+        else pre[p / 2] |= acc << 16;
+    }
 }
+
+// Prefix p of a stored table (tab points to the table's first byte).
+template <int M> __device__ __forceinline__ unsigned prefix_at(const void* tab, int p) {
+    if (M == 32) return static_cast<const unsigned*>(tab)[p];
+    return static_cast<const unsigned short*>(tab)[p];
+}
+
+// The first `cap` entries of `avail` (a set of positions of one line) in the line's sorted
+// order, or all of them if there are no more than `cap`: binary search for the shortest
+// prefix of the order that holds `cap` available entries.
 template <int M>
-__device__ __forceinline__ void store_tables(const unsigned (&packed)[M / 4], unsigned char* perm, unsigned char* rank) {
+__device__ __forceinline__ unsigned first_available(unsigned avail, int cap, const void* tab) {
+    if (__popc(avail) <= cap) return avail;
+    int p = 0;
 #pragma unroll
-    for (int w = 0; w < M / 4; ++w) reinterpret_cast<unsigned*>(perm)[w] = packed[w];
+    for (int b = M / 2; b > 0; b >>= 1)
+        if (__popc(avail & prefix_at<M>(tab, p + b - 1)) < cap) p += b;
+    return avail & prefix_at<M>(tab, p);
+}
+
+// Transpose of the M x M bit matrix whose row i is held by lane i of a group of M lanes
+// (bit j of x = element (i, j)): recursive exchange of the off-diagonal blocks.
+template <int M> __device__ __forceinline__ unsigned transpose_bits(unsigned x, int i) {
 #pragma unroll
-    for (int p = 0; p < M; ++p) rank[(packed[p / 4] >> (8 * (p % 4))) & 0xffu] = (unsigned char)p;
+    for (int s = M / 2; s > 0; s >>= 1) {
+        // positions whose bit s is clear
+        const unsigned lo = (s == 16) ? 0x0000ffffu : (s == 8) ? 0x00ff00ffu : (s == 4) ? 0x0f0f0f0fu
+                          : (s == 2) ? 0x33333333u : 0x55555555u;
+        const unsigned y = __shfl_xor_sync(FULL, x, s);
+        const bool up = (i & s) != 0;
+        const unsigned keep = up ? ~lo : lo;
+        const unsigned z = up ? (y >> s) : (y << s);
+        x = (x & keep) | (z & ~keep);
+    }
+    return x;
 }
 
 // Greedy selection + local search for the block of this lane's group.
 //   ks, ws: shared-memory pointers to element (0,0) of the block's keys and
-//   |scores| (row stride WS); the key cells are overwritten.  tb: the group's
-//   scratch; active: group has a block.
+//   |scores| (row stride WS); the key cells are overwritten.  cpre: this
+//   lane's column-prefix table when it does not fit in the key cells (M = 32).
+//   tb: the group's scratch; active: group has a block.
 // Returns this lane's row of the mask (M bits).  flags accumulates DEV_* bits.
 template <int M>
-__device__ __forceinline__ unsigned round_block(float* ks, const float* ws, RoundScratch<M>& tb, int lane,
-                                                bool active, int N, int ls_steps, int& flags) {
+__device__ __forceinline__ unsigned round_block(float* ks, const float* ws, unsigned* cpre, RoundScratch<M>& tb,
+                                                int lane, bool active, int N, int ls_steps, int& flags) {
     using G = Geom<M>;
     constexpr int WS = G::WS;
     constexpr unsigned GM = (M == 32) ? 0xffffffffu : ((1u << (M & 31)) - 1u);
     const int i = lane % M;            // my row, and my column
     const int gsh = (lane / M) * M;    // first lane of my group
 
-    // ---- sorted orders of my row and of my column (Algorithm 2 line 2)
-    unsigned char* const rperm = reinterpret_cast<unsigned char*>(ks + i * WS);
-    unsigned char* const cperm = rperm + M;
-    unsigned char* const rrank = rperm + 2 * M;
-    unsigned char* const crank = rperm + 3 * M;
+    // ---- sorted orders of my row and of my column (Algorithm 2 line 2), kept as prefix sets
+    unsigned char* const rtab = reinterpret_cast<unsigned char*>(ks + i * WS);
+    unsigned char* const ctab = (M == 32) ? reinterpret_cast<unsigned char*>(cpre) : rtab + 2 * M;
     {
-        unsigned pr[M / 4], pc[M / 4];
-        sort_line<M>(ks + i * WS, 1, pr);
+        constexpr int PW = PreWords<M>::value;
+        unsigned pc[PW];
         sort_line<M>(ks + i, WS, pc);
+        if (M == 32) {                      // not aliased with the keys: store at once
+#pragma unroll
+            for (int w = 0; w < PW; ++w) reinterpret_cast<unsigned*>(ctab)[w] = pc[w];
+        }
+        unsigned pr[PW];
+        sort_line<M>(ks + i * WS, 1, pr);
         __syncwarp();                       // every lane is done reading keys
-        store_tables<M>(pr, rperm, rrank);
-        store_tables<M>(pc, cperm, crank);
+#pragma unroll
+        for (int w = 0; w < PW; ++w) reinterpret_cast<unsigned*>(rtab)[w] = pr[w];
+        if (M != 32) {
+#pragma unroll
+            for (int w = 0; w < PW; ++w) reinterpret_cast<unsigned*>(ctab)[w] = pc[w];
+        }
     }
     __syncwarp();
 
     // ---- greedy selection (lines 3-6) in synchronous rounds.  An available
-    // entry (not taken, row and column not full) that ranks below the
-    // remaining capacity among the available entries of both its row and its
-    // column is taken by the sequential scan whatever happens elsewhere, so
-    // all such entries are taken at once; the first available entry in the
-    // global order always qualifies, hence every round makes progress and the
-    // fixed point is the sequential result.
-    unsigned A = active ? GM : 0u, B = A;   // available entries, rank space
+    // entry (not taken, row and column not full) that is among the first
+    // capR available entries of its row and the first capC of its column
+    // (cap = remaining capacity) is taken by the sequential scan whatever
+    // happens elsewhere, so all such entries are taken at once; the first
+    // available entry in the global order always qualifies, hence every round
+    // makes progress and the fixed point is the sequential result.  availR:
+    // available columns of my row; availC: available rows of my column.
+    unsigned availR = active ? GM : 0u, availC = availR;
     int capR = active ? N : 0, capC = capR;
-    bool rowdone = !active, coldone = !active;
     unsigned sel = 0u;
     for (int round = 0; round < M * M; ++round) {
-        if (!__any_sync(FULL, A != 0u)) break;
+        if (!__any_sync(FULL, availR != 0u)) break;
         if (round == M * M - 1) flags |= DEV_INTERNAL;
-        // picks: the first capR (capC) available entries in rank order
-        unsigned ar = A, bc = B, pickR = 0u, pickC = 0u, RS = 0u, CS = 0u;
-        int nr = capR, nc = capC;
-        while (__any_sync(FULL, (nr > 0 && ar) || (nc > 0 && bc))) {
-            if (nr > 0 && ar) {
-                const int p = __ffs(ar) - 1;
-                ar &= ar - 1; --nr;
-                pickR |= 1u << p;
-                RS |= 1u << rperm[p];
-            }
-            if (nc > 0 && bc) {
-                const int s = __ffs(bc) - 1;
-                bc &= bc - 1; --nc;
-                pickC |= 1u << s;
-                CS |= 1u << cperm[s];
-            }
-        }
-        tb.rs[i] = RS;
-        tb.cs[i] = CS;
-        __syncwarp();
+        const unsigned pickR = first_available<M>(availR, capR, rtab);
+        const unsigned pickC = first_available<M>(availC, capC, ctab);
         // an entry picked from both sides is taken
-        while (__any_sync(FULL, pickR | pickC)) {
-            if (pickR) {
-                const int p = __ffs(pickR) - 1;
-                pickR &= pickR - 1;
-                const int j = rperm[p];
-                if ((tb.cs[j] >> i) & 1u) { sel |= 1u << j; A &= ~(1u << p); --capR; }
-            }
-            if (pickC) {
-                const int s = __ffs(pickC) - 1;
-                pickC &= pickC - 1;
-                const int r = cperm[s];
-                if ((tb.rs[r] >> i) & 1u) { B &= ~(1u << s); --capC; }
-            }
-        }
-        __syncwarp();
+        const unsigned takenR = pickR & transpose_bits<M>(pickC, i);   // columns taken in my row
+        const unsigned takenC = transpose_bits<M>(takenR, i);          // rows taken in my column
+        sel |= takenR;
+        capR -= __popc(takenR);
+        capC -= __popc(takenC);
         // lines that just filled up drop out, and so do their entries
-        const bool rfull = (capR == 0) && !rowdone, cfull = (capC == 0) && !coldone;
-        unsigned nfr = (__ballot_sync(FULL, rfull) >> gsh) & GM;
-        unsigned nfc = (__ballot_sync(FULL, cfull) >> gsh) & GM;
-        if (rfull) { A = 0u; rowdone = true; }
-        if (cfull) { B = 0u; coldone = true; }
-        while (__any_sync(FULL, nfr | nfc)) {
-            if (nfr) {
-                const int r = __ffs(nfr) - 1;
-                nfr &= nfr - 1;
-                B &= ~(1u << crank[r]);
-            }
-            if (nfc) {
-                const int c = __ffs(nfc) - 1;
-                nfc &= nfc - 1;
-                A &= ~(1u << rrank[c]);
-            }
-        }
+        const unsigned fullR = (__ballot_sync(FULL, capR == 0) >> gsh) & GM;
+        const unsigned fullC = (__ballot_sync(FULL, capC == 0) >> gsh) & GM;
+        availR = (capR == 0) ? 0u : (availR & ~takenR & ~fullC);
+        availC = (capC == 0) ? 0u : (availC & ~takenC & ~fullR);
     }
 
     // ---- local search (lines 7-13, Eq. 6).  Lane j' scans i' = 0..M-1.
@@ -736,6 +738,7 @@ template <int M, int MODE> struct SmemLayout {
     float k[M * G::WS];
     RoundScratch<M> tb[WARPS * G::GPW];
     unsigned int bits[M * G::WORDS];
+    unsigned int cpre[(M == 32) ? WARPS * 32 * CPRE_STRIDE : 1];   // column-prefix tables (M = 32)
 };
 template <int M> struct SmemLayout<M, 1> {   // Algorithm 1 alone: score panel and the t0 stash
     using G = Geom<M>;
@@ -743,6 +746,7 @@ template <int M> struct SmemLayout<M, 1> {   // Algorithm 1 alone: score panel a
     float k[WARPS * 32 * Tile<M>::MR * Tile<M>::MC];
     RoundScratch<M> tb[1];
     unsigned int bits[1];
+    unsigned int cpre[1];
 };
 // Resident CTAs per SM the register allocation aims for.
 template <int M> struct MinBlocks { static constexpr int value = (M == 4) ? 5 : 4; };
@@ -869,7 +873,8 @@ __global__ void __launch_bounds__(WARPS * 32, MinBlocks<M>::value) tsenor_kernel
             const int blk = warp * G::BPW + pass * G::GPW + grp;
             const bool active = blk * M < valid_cols;
             const unsigned row_bits =
-                round_block<M>(sm.k + blk * M, sm.w + blk * M, tb, lane, active, P.N, P.ls_steps, flags);
+                round_block<M>(sm.k + blk * M, sm.w + blk * M, sm.cpre + (warp * 32 + lane) * CPRE_STRIDE, tb, lane,
+                               active, P.N, P.ls_steps, flags);
             if (active) {
                 const int off = blk * M;
                 if (M == 32) sm.bits[(lane % M) * G::WORDS + off / 32] = row_bits;
