@@ -32,9 +32,12 @@ SM_COUNT = 148
 FP32_LANES_PER_CLK_PER_SM = 128  # fp32 lane operations dispatched per clock per SM (4 x 32)
 XU_PER_CLK_PER_SM = 16          # special-function results per clock per SM
 NOMINAL_SM_MHZ = 1965.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one tsenor_kernel<32,0> launch on the
-# 14336x4096 matrix, from the ncu capture summarised under profiles/ (None until captured)
-NCU_DRAM_BYTES_PER_LAUNCH = 244.09e6   # 235.01 MB read + 9.09 MB written
+# Figures of one tsenor_kernel<32,0> launch on the 14336x4096 matrix taken from the ncu capture
+# summarised in PROFILE_SUMMARY (not measured by this script: they go stale if the kernel changes
+# and the capture is not repeated, which is why the JSON line names their source).
+PROFILE_SUMMARY = "profiles/tsenor_kernel_m32_solve_config4_up.md"
+NCU_DRAM_BYTES_PER_LAUNCH = 244.09e6      # dram__bytes_read.sum + dram__bytes_write.sum
+NCU_WARP_INST_PER_BLOCK_ITER = 170.0      # smsp__inst_executed.sum / (57,344 blocks x 300 iterations)
 
 
 def fp32_lane_ops_per_block(M, T):
@@ -212,10 +215,11 @@ def workload_config(workload, jobs):
            "blocks_per_step_per_gpu": sum(j.blocks for j in jobs), "iters": T_ITERS}
     if len({(j.N, j.M) for j in jobs}) == 1:
         cfg["M"], cfg["N"] = jobs[0].M, jobs[0].N
-    small = min(j.score_bytes for j in jobs) < 2 * 126e6
-    cfg["l2"] = ("a 256 MB buffer is overwritten between timed steps (inputs do not exceed the 126 MB L2); "
+    small = min(j.score_bytes for j in jobs) <= 126e6
+    cfg["l2"] = ("a 256 MB buffer is overwritten between timed steps (some input fits in the 126 MB L2); "
                  "value sums the per-step CUDA-event times" if small else
-                 "inputs (235 MB per matrix) exceed the 126 MB L2; no flush needed")
+                 f"every input ({min(j.score_bytes for j in jobs) / 1e6:.0f} MB or more per matrix) exceeds the "
+                 "126 MB L2 and consecutive launches read different matrices; no flush needed")
     return cfg, small
 
 
@@ -241,14 +245,33 @@ def oracle_sample(job, blocks_wanted):
     return np.ascontiguousarray(full[: nrows * M]), nrows * per_row, float(full.max())
 
 
-def time_oracle(job, blocks_wanted):
+def time_oracle(job, blocks_wanted, want_masks=False):
     import oracle
     sample, nblk, mx = oracle_sample(job, blocks_wanted)
     tau = synth.default_tau(mx)
     t0 = time.perf_counter()
-    oracle.solve(sample, job.N, job.M, tau, T_ITERS, LS_STEPS)
+    bits = oracle.solve(sample, job.N, job.M, tau, T_ITERS, LS_STEPS)
     dt = time.perf_counter() - t0
+    if want_masks:
+        return nblk / dt, nblk, dt, oracle.num_threads(), sample, bits
     return nblk / dt, nblk, dt, oracle.num_threads()
+
+
+def objective_parity(sample, oracle_bits, gpu_bits):
+    """Relative difference of the retained score of the CUDA mask and of the oracle's mask on the
+    rows the oracle solved (both objectives computed by the oracle's own fp64 sum)."""
+    import oracle
+    o_ref = oracle.objective(sample, oracle_bits)
+    o_gpu = oracle.objective(sample, np.ascontiguousarray(gpu_bits[: sample.shape[0]]))
+    return (o_gpu - o_ref) / o_ref, o_gpu, o_ref
+
+
+# One matrix per remaining pattern of the sweep, timed after the headline (outside its timed
+# region) so that the default run reports every N:M: config 2, a 4096x4096 matrix drawn like
+# config 1, and config 3.
+PATTERN_JOBS = (("2:4", lambda: synth.config(2)),
+                ("4:8", lambda: synth.Workload("config1-shaped-4096", synth.gaussian_abs(4096, 4096, 1.0, 1000), 4, 8)),
+                ("8:16", lambda: synth.config(3)))
 
 
 def run_reference(args, rank):
@@ -439,6 +462,29 @@ def run_cuda(args, rank, world, local_rank):
     barrier()
     e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
 
+    patterns = None
+    if rank == 0 and world == 1 and args.workload == "config4" and not args.no_patterns:
+        patterns = {}
+        if flush_buf is None:
+            flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        for label, make in PATTERN_JOBS:
+            w = make()
+            Wd = torch.from_numpy(w.scores).to(dev)
+            tau = synth.default_tau(float(ts.max_abs(Wd).item()))
+            pm = ts.new_mask(w.scores.shape[0], w.scores.shape[1], dev)
+            times = []
+            for k in range(3 + 5):
+                flush_buf.fill_(k)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                ts.solve(Wd, w.N, w.M, tau, T_ITERS, LS_STEPS, mask_out=pm, status=status)
+                b.record()
+                torch.cuda.synchronize()
+                if k >= 3:
+                    times.append(a.elapsed_time(b))
+            patterns[label] = (w, statistics.mean(times), int(ts.check(pm, *w.scores.shape, w.N, w.M).item()))
+            del Wd, pm
+
     if rank == 0:
         peaks, peak_kind = measured_peaks()
         sec = total_ms / 1e3
@@ -477,6 +523,10 @@ def run_cuda(args, rank, world, local_rank):
                 "kernel": "tsenor_kernel<M,0>" if len(jobs) > 2 else f"tsenor_kernel<{jobs[0].M},0>",
                 "launch_ms": 1e3 * solve_s / (args.steps * nj),
                 "traffic": NCU_DRAM_BYTES_PER_LAUNCH if args.workload == "config4" else None,
+                "traffic_source": (f"ncu capture of one launch on the 14336x4096 matrix, {PROFILE_SUMMARY} "
+                                   "(not measured in this run)") if args.workload == "config4" else None,
+                "warp_inst_per_block_iter": NCU_WARP_INST_PER_BLOCK_ITER if args.workload == "config4" else None,
+                "warp_inst_model_per_block_iter": 80.0 if args.workload == "config4" else None,
                 "algorithmic_bytes": alg_bytes / nj,
                 "hbm_frac": alg_bytes * args.steps / solve_s / 1e9 / peaks["hbm_gbs"],
                 # time the SFU alone would need for a log-domain iteration, over the measured time:
@@ -485,14 +535,37 @@ def run_cuda(args, rank, world, local_rank):
                 "vs_sfu_bound_paper_listing": t_sfu_lit / solve_s,
             },
         }
+        # spread of the fraction over the timed steps (each step = all launches of the step)
+        step_frac = sorted(sum(fp32_lane_ops_per_block(j.M, T_ITERS) * j.blocks for j in jobs) /
+                           (sum(row) / 1e3) / fp32_peak for row in launch_ms)
+        out["roofline"]["frac_median"] = statistics.median(step_frac)
+        out["roofline"]["frac_min"], out["roofline"]["frac_max"] = step_frac[0], step_frac[-1]
+        if patterns is not None:
+            pat = {f"{jobs[0].N}:{jobs[0].M}": {
+                "workload": "headline (both matrices)", "blocks_per_s": value,
+                "gb_scores_per_s": out["gb_scores_per_s"], "frac": achieved / fp32_peak, "infeasible_blocks": bad}}
+            for label, (w, ms, nbad) in patterns.items():
+                pat[label] = {
+                    "workload": f"{w.name} {w.scores.shape[0]}x{w.scores.shape[1]}", "ms_per_launch": ms,
+                    "blocks_per_s": w.blocks / (ms / 1e3),
+                    "gb_scores_per_s": w.scores.nbytes / (ms / 1e3) / 1e9,
+                    "frac": fp32_lane_ops_per_block(w.M, T_ITERS) * w.blocks / (ms / 1e3) / fp32_peak,
+                    "infeasible_blocks": nbad}
+            out["patterns"] = dict(sorted(pat.items(), key=lambda kv: int(kv[0].split(":")[1])))
+            out["patterns_note"] = ("one matrix per pattern, mean of 5 launches after 3 warm-up launches, "
+                                    "256 MB L2 flush before each, timed outside the headline region")
         if clocks and clocks.get("sm_mhz"):
             out["roofline"]["frac_at_sampled_clock"] = achieved / (fp32_peak * clocks["sm_mhz"] /
                                                                    peaks.get("sm_max_mhz", NOMINAL_SM_MHZ))
         if not args.no_cpu_baseline and world == 1:
-            rate, nblk, dt, cores = time_oracle(jobs[0], args.cpu_blocks)
+            rate, nblk, dt, cores, sample, obits = time_oracle(jobs[0], args.cpu_blocks, want_masks=True)
             out["cpu_baseline"] = {
                 "value": rate, "unit": "blocks/s", "cores": cores, "kind": "oracle",
                 "sample": f"first {nblk} blocks of {jobs[0].name}, {dt:.1f} s of oracle time"}
+            # the oracle's masks of that sample are kept: objective parity of the CUDA masks
+            rel, o_gpu, o_ref = objective_parity(sample, obits, djobs[0].result().cpu().numpy().view(np.uint32))
+            out["objective_rel_err"] = {"value": rel, "blocks": nblk, "of": jobs[0].name, "bound": 1e-4,
+                                        "objective_cuda": o_gpu, "objective_oracle": o_ref}
         else:
             out["cpu_baseline"] = None
         print(json.dumps(out), flush=True)
@@ -510,6 +583,8 @@ def main():
                     help="config4 is the headline; the others are the remaining configurations and modes")
     ap.add_argument("--cpu-blocks", type=int, default=57344, help="oracle sample size for cpu_baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-patterns", action="store_true",
+                    help="skip the per-pattern launches (2:4, 4:8, 8:16) that follow the headline")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

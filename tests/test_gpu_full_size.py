@@ -86,15 +86,46 @@ def test_config0_paper_table_shape_8_16():
     _check_full(wl.scores, wl.N, wl.M, 256, seed=0)
 
 
-@pytest.mark.parametrize("N,M", synth.NM_SWEEP)
-@pytest.mark.parametrize("name", ["k_proj", "down_proj"])
-def test_config5_outlier_columns(name, N, M):
-    wl = synth.llama_layer(name, N, M, scale_rows=512 if name == "down_proj" else 0)
-    W = wl.scores
-    # make sure blocks that contain an outlier column are among the sampled ones
-    colmax = W.max(0)
+def _outlier_blocks_first_block_row(W, M):
+    """Blocks of the first block row that contain an outlier column (config 5)."""
+    colmax = W[: 4 * M].max(0)
     out_cols = np.flatnonzero(colmax > 8 * np.median(colmax))
     assert len(out_cols) > 0
-    nbc = W.shape[1] // M
-    extra = [int((r // M) * nbc + c // M) for c in out_cols[:8] for r in (0, W.shape[0] - 1)]
-    _check_full(W, N, M, 128, seed=5, extra_blocks=extra)
+    return sorted({int(c // M) for c in out_cols})
+
+
+@pytest.mark.parametrize("N,M", synth.NM_SWEEP)
+@pytest.mark.parametrize("name", list(synth.LLAMA3_8B_LAYER_SHAPES))
+def test_config5_every_shape_every_pattern_full_size(name, N, M):
+    """Config 5, layer 0: each of the seven linear shapes at its full size under each of the four
+    patterns.  Every block is checked for feasibility on the device; 128 random blocks plus every
+    block of the first block row that holds an outlier column go through the oracle."""
+    wl = synth.llama_layer(name, N, M)
+    W = wl.scores
+    assert W.shape == synth.LLAMA3_8B_LAYER_SHAPES[name]
+    _check_full(W, N, M, 128, seed=5, extra_blocks=_outlier_blocks_first_block_row(W, M))
+
+
+@pytest.mark.parametrize("layer", [1, 31])
+def test_config5_other_layers_q_proj_16_32(layer):
+    """The layer index only changes the seed: two more layers of the sweep for one shape."""
+    wl = synth.llama_layer("q_proj", 16, 32, layer=layer)
+    assert not np.array_equal(wl.scores[:64], synth.llama_layer("q_proj", 16, 32).scores[:64])
+    _check_full(wl.scores, 16, 32, 128, seed=50 + layer,
+                extra_blocks=_outlier_blocks_first_block_row(wl.scores, 32))
+
+
+@pytest.mark.parametrize("cfg,part", [(4, "up"), (3, "up"), (1, "up")])
+def test_whole_matrix_objective_against_the_oracle(cfg, part):
+    """The retained-score objective of the whole matrix (every block solved by the oracle, not
+    a sample): within 1e-4 relative, and the masks of at least 98 % of the blocks identical."""
+    wl = synth.config(cfg, part=part)
+    W, N, M = wl.scores, wl.N, wl.M
+    rows, cols = W.shape
+    tau = synth.default_tau(float(W.max()))
+    got = _bits(ts.solve(torch.from_numpy(W).to(DEV), N, M, tau, 300, -1))
+    want = oracle.solve(W, N, M, tau, 300)
+    o_gpu, o_ref = oracle.objective(W, got), oracle.objective(W, want)
+    assert abs(o_gpu - o_ref) <= OBJ_RTOL * o_ref, (o_gpu, o_ref)
+    differ = oracle.unpack_mask(got ^ want, cols).reshape(rows // M, M, cols // M, M).any(axis=(1, 3))
+    assert differ.mean() <= 0.02

@@ -79,6 +79,39 @@ def test_random_solve_cases_match_the_oracle(seed):
             # the greedy order among them is decided by noise (exact ties in fp64, 1e-7 apart in
             # fp32) and masks legitimately differ; the objective is compared once the plan has
             # separated, as at the method's operating point T = 300.
+            # These matrices hold a few dozen blocks, so one block that legitimately differs moves
+            # the total by more than 1e-4: 2e-3 here; the stated 1e-4 per matrix is held on the
+            # matrices of >= 1024 blocks below.
             want = oracle.solve(W, N, M, tau, iters)
             o_gpu, o_ref = oracle.objective(W, got), oracle.objective(W, want)
-            assert abs(o_gpu - o_ref) <= 2e-3 * o_ref, (seed, M, N, rows, cols, iters)
+            assert abs(o_gpu - o_ref) <= 2e-3 * o_ref, ("bound 2e-3 (small matrix)", seed, M, N, rows, cols, iters)
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_matrices_of_1024_blocks_or_more_hold_the_stated_bounds(seed):
+    """At the operating point (T = 300) and with at least 1024 blocks per matrix the stated bounds
+    apply as they are: plan within 1e-4, per-matrix objective within 1e-4 relative."""
+    rng = np.random.default_rng(7100 + seed)
+    M = [4, 8, 16, 32][seed % 4]
+    N = M // 2 if seed < 4 else int(rng.integers(1, M))
+    nbr, nbc = int(rng.integers(16, 40)), int(rng.integers(64, 80))
+    rows, cols = M * nbr, M * nbc
+    assert nbr * nbc >= 1024
+    kind = int(rng.integers(0, 3))
+    if kind == 0:
+        W = np.abs(rng.standard_normal((rows, cols))) * 0.02
+    elif kind == 1:
+        W = np.abs(rng.standard_t(3.0, (rows, cols))) * 0.0115
+    else:
+        W = np.abs(rng.standard_normal((rows, cols))) * 0.02 * np.where(rng.random(cols) < 0.01, 20.0, 1.0)[None, :]
+    W = W.astype(np.float32)
+    tau = float(rng.choice([50.0, 200.0]) / W.max())
+    Wd = torch.from_numpy(W).to(DEV)
+    st = ts.new_status(DEV)
+    plan = ts.dykstra(Wd, N, M, tau, 300, status=st).cpu().numpy()
+    assert np.abs(plan - oracle.dykstra(W, N, M, tau, 300)).max() <= 1e-4, ("bound 1e-4 (plan)", seed, M, N)
+    got = _bits(ts.solve(Wd, N, M, tau, 300, status=st))
+    assert int(st.item()) == 0
+    assert oracle.count_infeasible(got, rows, cols, N, M) == 0
+    o_gpu, o_ref = oracle.objective(W, got), oracle.objective(W, oracle.solve(W, N, M, tau, 300))
+    assert abs(o_gpu - o_ref) <= 1e-4 * o_ref, ("bound 1e-4 (objective)", seed, M, N, rows, cols, kind)
