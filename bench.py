@@ -144,7 +144,8 @@ def aggregate_rate(units_per_rank_per_step, steps, world, elapsed_ms):
     return world * units_per_rank_per_step * steps / (elapsed_ms / 1e3)
 
 
-WORKLOADS = ("config4", "config0", "config1", "config2", "config3", "config5", "admm", "wanda", "sparsegpt")
+WORKLOADS = ("config4", "config0", "config1", "config2", "config3", "config5", "admm", "admm_small", "wanda",
+             "sparsegpt")
 
 
 class Job:
@@ -164,7 +165,13 @@ def make_jobs(workload, index):
     if workload == "config4":
         return [Job(w.name, w.N, w.M, {"w": w.scores})
                 for w in (synth.config(4, index=index, part="up"), synth.config(4, index=index, part="down"))]
-    if workload in ("config0", "config1", "config2", "config3"):
+    if workload == "config1":     # 16 different matrices per step: a single 50 us launch between two
+        jobs = []                 # event records would time the host's launch path, not the kernel
+        for k in range(16):
+            w = synth.config(1, index=16 * index + k)
+            jobs.append(Job(f"{w.name}#{k}", w.N, w.M, {"w": w.scores}))
+        return jobs
+    if workload in ("config0", "config2", "config3"):
         w = synth.config(int(workload[-1]), index=index)
         return [Job(w.name, w.N, w.M, {"w": w.scores})]
     if workload == "config5":     # one decoder layer, every linear shape, the four patterns
@@ -178,6 +185,13 @@ def make_jobs(workload, index):
         W = (rng.standard_normal((14336, 4096), dtype=np.float32) * np.float32(0.02))
         V = (rng.standard_normal((14336, 4096), dtype=np.float32) * np.float32(0.004))
         return [Job("admm-up-16:32", 16, 32, {"w": W, "v": V}, kind="admm", scalar=1.0 / 0.3)]
+    if workload == "admm_small":  # the same on a small layer: the solver is called once per ADMM iteration
+        jobs = []
+        for k in range(8):
+            W = (rng.standard_normal((1024, 1024), dtype=np.float32) * np.float32(0.02))
+            V = (rng.standard_normal((1024, 1024), dtype=np.float32) * np.float32(0.004))
+            jobs.append(Job(f"admm-1024-8:16#{k}", 8, 16, {"w": W, "v": V}, kind="admm", scalar=1.0 / 0.3))
+        return jobs
     if workload == "wanda":       # config 3 with the score computed in the loader from bf16 weights
         import torch
         W = torch.from_numpy(rng.standard_normal((4096, 4096), dtype=np.float32) * np.float32(0.02)).to(torch.bfloat16)
@@ -193,17 +207,23 @@ def make_jobs(workload, index):
     raise ValueError(workload)
 
 
+GRAPH_WORKLOADS = ("config1", "admm_small", "sparsegpt")
+
 WORKLOAD_TEXT = {
     "config4": "config 4: Llama-3-8B MLP pair, up 14336x4096 + down 4096x14336, transposable 16:32, "
                "Student-t(3) scores std 0.02",
     "config0": "8192x8192 |N(0,0.02^2)|, 8:16 (shape of the paper's runtime tables)",
-    "config1": "config 1: 512x512 |N(0,1)|, 4:8 (latency case: 4096 blocks)",
+    "config1": "config 1: 512x512 |N(0,1)|, 4:8 (latency case: 4096 blocks per matrix); 16 different matrices "
+               "per step, launches back to back",
     "config2": "config 2: 4096x4096 |N(0,0.02^2)|, 2:4",
     "config3": "config 3: 4096x4096 Wanda-style scores, 8:16",
     "config5": "config 5: the 7 linear shapes of one Llama-3-8B layer, |N(0,0.02^2)| with 0.1% outlier columns x20, "
                "patterns 2:4, 4:8, 8:16, 16:32 (28 solves per step)",
     "admm": "ADMM D-update on 14336x4096: scores (W+V/rho)^2 computed in the loader, 16:32, then the "
             "keep-previous-mask safeguard",
+    "admm_small": "ADMM D-update on 1024x1024 layers (latency case: 4096 blocks per matrix): scores (W+V/rho)^2 "
+                  "computed in the loader, 8:16, then the keep-previous-mask safeguard; 8 different layers per step, "
+                  "launches back to back",
     "wanda": "Wanda scores |W_ij| a_j computed in the loader from bf16 W (4096x4096) and fp32 a_j, 8:16",
     "sparsegpt": "SparseGPT column groups: eight 14336x32 slabs solved one after the other (latency case: 448 "
                  "blocks per call), scores |W_ij / d_j| computed in the loader, 16:32",
@@ -215,6 +235,7 @@ def workload_config(workload, jobs):
            "blocks_per_step_per_gpu": sum(j.blocks for j in jobs), "iters": T_ITERS}
     if len({(j.N, j.M) for j in jobs}) == 1:
         cfg["M"], cfg["N"] = jobs[0].M, jobs[0].N
+    cfg["solves_per_step"] = len(jobs)
     small = min(j.score_bytes for j in jobs) <= 126e6
     cfg["l2"] = ("a 256 MB buffer is overwritten between timed steps (some input fits in the 126 MB L2); "
                  "value sums the per-step CUDA-event times" if small else
@@ -362,14 +383,15 @@ def run_cuda(args, rank, world, local_rank):
             else:
                 ts.solve_scores(src, j.N, j.M, self.tau, T_ITERS, LS_STEPS, mask_out=self.mask, status=status,
                                 stream=stream)
-            if j.kind == "admm":          # safeguard against the mask of the previous step
+            if j.kind == "admm":          # safeguard against the mask kept by the previous step
                 if self.have_prev:
                     ts.keep_better(src, self.prev, self.mask, self.obj2, stream=stream)
-                self.prev, self.mask = self.mask, self.prev
+                with torch.cuda.stream(stream or torch.cuda.current_stream()):
+                    self.prev.copy_(self.mask, non_blocking=True)
                 self.have_prev = True
 
         def result(self):
-            return self.prev if self.job.kind == "admm" else self.mask
+            return self.mask
 
     djobs = [DevJob(j) for j in jobs]
     blocks_per_step = sum(j.blocks for j in jobs)
@@ -386,6 +408,20 @@ def run_cuda(args, rank, world, local_rank):
             d.solve(d.res, d.src_res)
     barrier()
 
+    # Latency workloads (tens of microseconds per launch): one step is captured in a CUDA graph
+    # and replayed, so that the timed region holds the kernels and not the host's launch path.
+    graph, launches_per_replay = None, 0
+    if args.workload in GRAPH_WORKLOADS and not args.no_graph:
+        n_cap = ts.launch_count()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for d in djobs:
+                d.solve(d.res, d.src_res)
+        launches_per_replay = ts.launch_count() - n_cap
+        graph.replay()
+        barrier()
+        cfg["launch"] = "one step captured in a CUDA graph and replayed"
+
     # ---- timed region: inputs resident in HBM
     sampler = ClockSampler(local_rank) if rank == 0 else None
     n0 = ts.launch_count()
@@ -397,14 +433,21 @@ def run_cuda(args, rank, world, local_rank):
         if flush_buf is not None:
             flush_buf.fill_(s_ & 0xff)
         ev[s_][0].record()
+        if graph is not None:
+            graph.replay()
+            ev[s_][nj].record()
+            continue
         for k, d in enumerate(djobs):
             d.solve(d.res, d.src_res)
             ev[s_][k + 1].record()
     t_end.record()
     barrier()
-    launches = ts.launch_count() - n0
+    launches = ts.launch_count() - n0 + launches_per_replay * args.steps
     clocks = sampler.stop() if sampler else None
-    launch_ms = [[ev[s_][k].elapsed_time(ev[s_][k + 1]) for k in range(nj)] for s_ in range(args.steps)]
+    if graph is not None:    # no events inside a replay: the step's time, spread evenly over its launches
+        launch_ms = [[ev[s_][0].elapsed_time(ev[s_][nj]) / nj] * nj for s_ in range(args.steps)]
+    else:
+        launch_ms = [[ev[s_][k].elapsed_time(ev[s_][k + 1]) for k in range(nj)] for s_ in range(args.steps)]
     if flush_buf is not None:
         total_ms = sum(sum(row) for row in launch_ms)
     else:
@@ -583,6 +626,8 @@ def main():
                     help="config4 is the headline; the others are the remaining configurations and modes")
     ap.add_argument("--cpu-blocks", type=int, default=57344, help="oracle sample size for cpu_baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true",
+                    help="latency workloads: launch every solve from the host instead of replaying a CUDA graph")
     ap.add_argument("--no-patterns", action="store_true",
                     help="skip the per-pattern launches (2:4, 4:8, 8:16) that follow the headline")
     args = ap.parse_args()

@@ -223,6 +223,21 @@ int tsenor_last_cuda_error(void);
 /* Kernels launched by this library (all threads) since it was loaded. */
 int64_t tsenor_launch_count(void);
 
+/*
+ * Register layout of the Dykstra stage (Algorithm 1).  The kernels come in a throughput
+ * layout (fewest exchanges between lanes per element; for matrices with enough blocks to
+ * fill the GPU) and, for M < 32, a latency layout (every block spread over M lanes: a
+ * shorter chain of dependent work per iteration and more warps for the same matrix; for
+ * small matrices such as the per-iteration solves of the ADMM integration, Section 4).
+ * TSENOR_LAYOUT_AUTO (the default) picks the latency layout when even its finer panels
+ * give no more than four CTAs per SM.  The two layouts add the same numbers in a different
+ * order, so plans agree to rounding level (both within the documented 1e-4 of the fp64
+ * result), not bit for bit.  Process-wide setting, meant for tests and benchmarks; returns
+ * the previous value, or TSENOR_ERR_ARG.
+ */
+enum { TSENOR_LAYOUT_AUTO = 0, TSENOR_LAYOUT_THROUGHPUT = 1, TSENOR_LAYOUT_LATENCY = 2 };
+int tsenor_set_layout(int layout);
+
 #ifdef __cplusplus
 }
 #endif

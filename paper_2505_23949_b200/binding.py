@@ -21,8 +21,9 @@ EXPORTS = (
     "tsenor_solve", "tsenor_dykstra", "tsenor_round", "tsenor_objective", "tsenor_check",
     "tsenor_max_abs", "tsenor_mask_words_per_row", "tsenor_strerror", "tsenor_last_cuda_error",
     "tsenor_launch_count", "tsenor_solve_scores", "tsenor_scores_max", "tsenor_scores_materialize",
-    "tsenor_keep_better", "tsenor_simple_round", "tsenor_dykstra_scores",
+    "tsenor_keep_better", "tsenor_simple_round", "tsenor_dykstra_scores", "tsenor_set_layout",
 )
+LAYOUT_AUTO, LAYOUT_THROUGHPUT, LAYOUT_LATENCY = 0, 1, 2
 
 SCORES_ABS, SCORES_ADMM, SCORES_COLDIV, SCORES_COLMUL = 0, 1, 2, 3
 
@@ -81,6 +82,8 @@ def lib():
         L.tsenor_strerror.restype = C.c_char_p
         L.tsenor_launch_count.argtypes = []
         L.tsenor_launch_count.restype = i64
+        L.tsenor_set_layout.argtypes = [i32]
+        L.tsenor_set_layout.restype = i32
         _lib = L
     return _lib
 
@@ -103,6 +106,36 @@ def _ptr(t):
     return None if t is None else C.c_void_p(t.data_ptr())
 
 
+def _out(t, name, dtype, device, shape=None, min_numel=None):
+    """Checks a caller-supplied output (or status / scratch) tensor before its pointer goes to
+    the library: a wrong dtype, shape, layout or device would become an out-of-bounds write
+    on the GPU.  None passes through (the argument is optional or allocated by the caller)."""
+    if t is None:
+        return None
+    if not (isinstance(t, torch.Tensor) and t.is_cuda):
+        raise TypeError(f"{name} must be a CUDA tensor")
+    if t.dtype != dtype:
+        raise TypeError(f"{name} must have dtype {dtype}, not {t.dtype}")
+    if t.device != torch.device(device):
+        raise ValueError(f"{name} is on {t.device}, the input on {torch.device(device)}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name} must have shape {tuple(shape)}, not {tuple(t.shape)}")
+    if min_numel is not None and t.numel() < min_numel:
+        raise ValueError(f"{name} needs at least {min_numel} element(s)")
+    return t
+
+
+def _mask_out(t, rows, cols, device, name="mask_out"):
+    return _out(t, name, torch.int32, device, shape=(rows, mask_words_per_row(cols)))
+
+
+def _on(device):
+    """Makes the tensors' device current around a call: the library launches on the current device."""
+    return torch.cuda.device(torch.device(device))
+
+
 def mask_words_per_row(cols):
     return int(lib().tsenor_mask_words_per_row(int(cols)))
 
@@ -119,13 +152,24 @@ def launch_count():
     return int(lib().tsenor_launch_count())
 
 
+def set_layout(layout):
+    """tsenor_set_layout: LAYOUT_AUTO / LAYOUT_THROUGHPUT / LAYOUT_LATENCY; returns the previous one."""
+    rc = lib().tsenor_set_layout(int(layout))
+    if rc < 0:
+        raise TsenorError(rc, "tsenor_set_layout")
+    return rc
+
+
 def solve(scores, N, M, tau, iters=300, ls_steps=-1, mask_out=None, status=None, stream=None):
     """tsenor_solve: Algorithm 1 + Algorithm 2 on every M x M block.  Asynchronous."""
     p, rows, cols, ld = _mat(scores, "scores")
     if mask_out is None:
         mask_out = new_mask(rows, cols, scores.device)
-    rc = lib().tsenor_solve(p, rows, cols, ld, int(N), int(M), float(tau), int(iters), int(ls_steps),
-                            _ptr(mask_out), _ptr(status), _stream(stream))
+    _mask_out(mask_out, rows, cols, scores.device)
+    _out(status, "status", torch.int32, scores.device, min_numel=1)
+    with _on(scores.device):
+        rc = lib().tsenor_solve(p, rows, cols, ld, int(N), int(M), float(tau), int(iters), int(ls_steps),
+                                _ptr(mask_out), _ptr(status), _stream(stream))
     if rc:
         raise TsenorError(rc, "tsenor_solve")
     return mask_out
@@ -136,9 +180,13 @@ def dykstra(scores, N, M, tau, iters=300, plan_is_log=False, plan_out=None, stat
     p, rows, cols, ld = _mat(scores, "scores")
     if plan_out is None:
         plan_out = torch.empty((rows, cols), dtype=torch.float32, device=scores.device)
-    pp, _, _, ldp = _mat(plan_out, "plan_out")
-    rc = lib().tsenor_dykstra(p, rows, cols, ld, int(N), int(M), float(tau), int(iters), pp, ldp,
-                              int(bool(plan_is_log)), _ptr(status), _stream(stream))
+    pp, pr, pc, ldp = _mat(plan_out, "plan_out")
+    if (pr, pc) != (rows, cols) or plan_out.device != scores.device:
+        raise ValueError("plan_out must have the shape and device of scores")
+    _out(status, "status", torch.int32, scores.device, min_numel=1)
+    with _on(scores.device):
+        rc = lib().tsenor_dykstra(p, rows, cols, ld, int(N), int(M), float(tau), int(iters), pp, ldp,
+                                  int(bool(plan_is_log)), _ptr(status), _stream(stream))
     if rc:
         raise TsenorError(rc, "tsenor_dykstra")
     return plan_out
@@ -150,10 +198,15 @@ def round_plan(plan_key, scores, N, M, ls_steps=-1, mask_out=None, status=None, 
     ps, r2, c2, ld = _mat(scores, "scores")
     if (rows, cols) != (r2, c2):
         raise ValueError("plan_key and scores differ in shape")
+    if plan_key.device != scores.device:
+        raise ValueError("plan_key and scores are on different devices")
     if mask_out is None:
         mask_out = new_mask(rows, cols, scores.device)
-    rc = lib().tsenor_round(pk, ldk, ps, ld, rows, cols, int(N), int(M), int(ls_steps),
-                            _ptr(mask_out), _ptr(status), _stream(stream))
+    _mask_out(mask_out, rows, cols, scores.device)
+    _out(status, "status", torch.int32, scores.device, min_numel=1)
+    with _on(scores.device):
+        rc = lib().tsenor_round(pk, ldk, ps, ld, rows, cols, int(N), int(M), int(ls_steps),
+                                _ptr(mask_out), _ptr(status), _stream(stream))
     if rc:
         raise TsenorError(rc, "tsenor_round")
     return mask_out
@@ -164,7 +217,10 @@ def objective(scores, mask, out=None, stream=None):
     p, rows, cols, ld = _mat(scores, "scores")
     if out is None:
         out = torch.empty(1, dtype=torch.float64, device=scores.device)
-    rc = lib().tsenor_objective(p, ld, _ptr(mask), rows, cols, _ptr(out), _stream(stream))
+    _mask_out(mask, rows, cols, scores.device, "mask")
+    _out(out, "out", torch.float64, scores.device, min_numel=1)
+    with _on(scores.device):
+        rc = lib().tsenor_objective(p, ld, _ptr(mask), rows, cols, _ptr(out), _stream(stream))
     if rc:
         raise TsenorError(rc, "tsenor_objective")
     return out
@@ -172,9 +228,14 @@ def objective(scores, mask, out=None, stream=None):
 
 def check(mask, rows, cols, N, M, out=None, stream=None):
     """tsenor_check: 1-element int64 device tensor with the number of infeasible blocks."""
+    if not (isinstance(mask, torch.Tensor) and mask.is_cuda):
+        raise TypeError("mask must be a CUDA tensor")
     if out is None:
         out = torch.empty(1, dtype=torch.int64, device=mask.device)
-    rc = lib().tsenor_check(_ptr(mask), int(rows), int(cols), int(N), int(M), _ptr(out), _stream(stream))
+    _mask_out(mask, int(rows), int(cols), mask.device, "mask")
+    _out(out, "out", torch.int64, mask.device, min_numel=1)
+    with _on(mask.device):
+        rc = lib().tsenor_check(_ptr(mask), int(rows), int(cols), int(N), int(M), _ptr(out), _stream(stream))
     if rc:
         raise TsenorError(rc, "tsenor_check")
     return out
@@ -185,7 +246,9 @@ def max_abs(scores, out=None, stream=None):
     p, rows, cols, ld = _mat(scores, "scores")
     if out is None:
         out = torch.empty(1, dtype=torch.float32, device=scores.device)
-    rc = lib().tsenor_max_abs(p, rows, cols, ld, _ptr(out), _stream(stream))
+    _out(out, "out", torch.float32, scores.device, min_numel=1)
+    with _on(scores.device):
+        rc = lib().tsenor_max_abs(p, rows, cols, ld, _ptr(out), _stream(stream))
     if rc:
         raise TsenorError(rc, "tsenor_max_abs")
     return out
@@ -210,14 +273,14 @@ class Scores:
         d.ld = w.stride(0) if self.rows > 1 else max(w.stride(0), self.cols)
         if v is not None:
             _, r2, c2, ldv = _mat(v, "v")
-            if (r2, c2) != (self.rows, self.cols):
-                raise ValueError("v and w differ in shape")
+            if (r2, c2) != (self.rows, self.cols) or v.device != w.device:
+                raise ValueError("v and w differ in shape or device")
             d.v, d.ld_v = v.data_ptr(), ldv
         d.scalar = float(scalar)
         if colvec is not None:
             if not (colvec.is_cuda and colvec.dtype == torch.float32 and colvec.is_contiguous()
-                    and colvec.numel() == self.cols):
-                raise TypeError("colvec must be a contiguous float32 CUDA vector of length cols")
+                    and colvec.numel() == self.cols and colvec.device == w.device):
+                raise TypeError("colvec must be a contiguous float32 CUDA vector of length cols on w's device")
             d.colvec = colvec.data_ptr()
         d.per_block_tau = int(bool(per_block_tau))
         self.desc = d
@@ -231,8 +294,11 @@ def solve_scores(src, N, M, tau, iters=300, ls_steps=-1, mask_out=None, status=N
     """tsenor_solve_scores: the whole method on a described score matrix."""
     if mask_out is None:
         mask_out = new_mask(src.rows, src.cols, src.device)
-    rc = lib().tsenor_solve_scores(C.byref(src.desc), src.rows, src.cols, int(N), int(M), float(tau), int(iters),
-                                   int(ls_steps), _ptr(mask_out), _ptr(status), _stream(stream))
+    _mask_out(mask_out, src.rows, src.cols, src.device)
+    _out(status, "status", torch.int32, src.device, min_numel=1)
+    with _on(src.device):
+        rc = lib().tsenor_solve_scores(C.byref(src.desc), src.rows, src.cols, int(N), int(M), float(tau), int(iters),
+                                       int(ls_steps), _ptr(mask_out), _ptr(status), _stream(stream))
     if rc:
         raise TsenorError(rc, "tsenor_solve_scores")
     return mask_out
@@ -242,9 +308,13 @@ def dykstra_scores(src, N, M, tau, iters=300, plan_is_log=False, plan_out=None, 
     """tsenor_dykstra_scores: Algorithm 1 only on a described score matrix."""
     if plan_out is None:
         plan_out = torch.empty((src.rows, src.cols), dtype=torch.float32, device=src.device)
-    pp, _, _, ldp = _mat(plan_out, "plan_out")
-    rc = lib().tsenor_dykstra_scores(C.byref(src.desc), src.rows, src.cols, int(N), int(M), float(tau), int(iters),
-                                     pp, ldp, int(bool(plan_is_log)), _ptr(status), _stream(stream))
+    pp, pr, pc, ldp = _mat(plan_out, "plan_out")
+    if (pr, pc) != (src.rows, src.cols) or plan_out.device != src.device:
+        raise ValueError("plan_out must have the shape and device of the score source")
+    _out(status, "status", torch.int32, src.device, min_numel=1)
+    with _on(src.device):
+        rc = lib().tsenor_dykstra_scores(C.byref(src.desc), src.rows, src.cols, int(N), int(M), float(tau),
+                                         int(iters), pp, ldp, int(bool(plan_is_log)), _ptr(status), _stream(stream))
     if rc:
         raise TsenorError(rc, "tsenor_dykstra_scores")
     return plan_out
@@ -254,7 +324,9 @@ def scores_max(src, out=None, stream=None):
     """tsenor_scores_max: 1-element float32 device tensor with the largest score."""
     if out is None:
         out = torch.empty(1, dtype=torch.float32, device=src.device)
-    rc = lib().tsenor_scores_max(C.byref(src.desc), src.rows, src.cols, _ptr(out), _stream(stream))
+    _out(out, "out", torch.float32, src.device, min_numel=1)
+    with _on(src.device):
+        rc = lib().tsenor_scores_max(C.byref(src.desc), src.rows, src.cols, _ptr(out), _stream(stream))
     if rc:
         raise TsenorError(rc, "tsenor_scores_max")
     return out
@@ -264,8 +336,11 @@ def scores_materialize(src, out=None, stream=None):
     """tsenor_scores_materialize: the described scores as a float32 matrix."""
     if out is None:
         out = torch.empty((src.rows, src.cols), dtype=torch.float32, device=src.device)
-    p, _, _, ld = _mat(out, "out")
-    rc = lib().tsenor_scores_materialize(C.byref(src.desc), src.rows, src.cols, p, ld, _stream(stream))
+    p, orows, ocols, ld = _mat(out, "out")
+    if (orows, ocols) != (src.rows, src.cols) or out.device != src.device:
+        raise ValueError("out must have the shape and device of the score source")
+    with _on(src.device):
+        rc = lib().tsenor_scores_materialize(C.byref(src.desc), src.rows, src.cols, p, ld, _stream(stream))
     if rc:
         raise TsenorError(rc, "tsenor_scores_materialize")
     return out
@@ -276,8 +351,12 @@ def keep_better(src, prev_mask, mask_inout, obj2_out=None, stream=None):
     Returns the 2-element float64 device tensor {objective(new), objective(previous)}."""
     if obj2_out is None:
         obj2_out = torch.empty(2, dtype=torch.float64, device=src.device)
-    rc = lib().tsenor_keep_better(C.byref(src.desc), src.rows, src.cols, _ptr(prev_mask), _ptr(mask_inout),
-                                  _ptr(obj2_out), _stream(stream))
+    _mask_out(prev_mask, src.rows, src.cols, src.device, "prev_mask")
+    _mask_out(mask_inout, src.rows, src.cols, src.device, "mask_inout")
+    _out(obj2_out, "obj2_out", torch.float64, src.device, min_numel=2)
+    with _on(src.device):
+        rc = lib().tsenor_keep_better(C.byref(src.desc), src.rows, src.cols, _ptr(prev_mask), _ptr(mask_inout),
+                                      _ptr(obj2_out), _stream(stream))
     if rc:
         raise TsenorError(rc, "tsenor_keep_better")
     return obj2_out
@@ -288,7 +367,9 @@ def simple_round(plan_key, N, M, mask_out=None, stream=None):
     pk, rows, cols, ldk = _mat(plan_key, "plan_key")
     if mask_out is None:
         mask_out = new_mask(rows, cols, plan_key.device)
-    rc = lib().tsenor_simple_round(pk, ldk, rows, cols, int(N), int(M), _ptr(mask_out), _stream(stream))
+    _mask_out(mask_out, rows, cols, plan_key.device)
+    with _on(plan_key.device):
+        rc = lib().tsenor_simple_round(pk, ldk, rows, cols, int(N), int(M), _ptr(mask_out), _stream(stream))
     if rc:
         raise TsenorError(rc, "tsenor_simple_round")
     return mask_out

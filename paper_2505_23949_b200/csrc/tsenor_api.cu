@@ -70,25 +70,46 @@ int make_source(const tsenor_scores_t* d, int64_t cols, tsenor::ScoreSrc* out) {
     return TSENOR_OK;
 }
 
-template <int M, int MODE>
-int launch(const tsenor::Params& P, cudaStream_t st) {
-    using G = tsenor::Geom<M>;
-    // a slab (single block column) is cut into panels of vertically stacked blocks
-    const bool tall = (P.cols == M) && (P.rows > M);
+std::atomic<int> g_layout{TSENOR_LAYOUT_AUTO};
+
+// Panels (= CTAs) a matrix is cut into under layout V.
+template <int M, int V>
+int64_t panel_count(const tsenor::Params& P, bool tall, int64_t* npc_out) {
+    using G = tsenor::Geom<M, V>;
     constexpr int NB = G::PANEL / M;
     const int64_t npc = (P.cols + G::PANEL - 1) / G::PANEL;
-    const int64_t panels = tall ? (P.rows / M + NB - 1) / NB : (P.rows / M) * npc;
+    *npc_out = npc;
+    return tall ? (P.rows / M + NB - 1) / NB : (P.rows / M) * npc;
+}
+
+int sm_count() {
+    static thread_local int cached_dev = -1, cached = 148;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev != cached_dev) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) cached = n;
+        cached_dev = dev;
+    }
+    return cached;
+}
+
+template <int M, int MODE, int V>
+int launch_layout(const tsenor::Params& P, bool tall, cudaStream_t st) {
+    using G = tsenor::Geom<M, V>;
+    int64_t npc = 0;
+    const int64_t panels = panel_count<M, V>(P, tall, &npc);
     if (panels == 0) return TSENOR_OK;
     if (panels > 0x7fffffffLL) return TSENOR_ERR_SHAPE;
     tsenor::Params Q = P;
     Q.npc = (int)npc;
     Q.tall = tall ? 1 : 0;
-    const size_t smem = sizeof(tsenor::SmemLayout<M, MODE>);
+    const size_t smem = sizeof(tsenor::SmemLayout<G, MODE>);
     static thread_local int configured_device = -1;
     int dev = 0;
     cudaGetDevice(&dev);
     if (configured_device != dev) {
-        cudaError_t e = cudaFuncSetAttribute(tsenor::tsenor_kernel<M, MODE>,
+        cudaError_t e = cudaFuncSetAttribute(tsenor::tsenor_kernel<M, MODE, V>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) {
             g_last_cuda_error = (int)e;
@@ -96,8 +117,27 @@ int launch(const tsenor::Params& P, cudaStream_t st) {
         }
         configured_device = dev;
     }
-    tsenor::tsenor_kernel<M, MODE><<<(unsigned)panels, tsenor::WARPS * 32, smem, st>>>(Q);
+    tsenor::tsenor_kernel<M, MODE, V><<<(unsigned)panels, tsenor::WARPS * 32, smem, st>>>(Q);
     return finish_launch();
+}
+
+// Chooses the register layout: the latency layout (a block over M lanes) when even its
+// finer panels leave the GPU with no more than four CTAs per SM, i.e. when the run time is
+// the chain of dependent iterations of a single warp rather than instruction throughput.
+template <int M, int MODE>
+int launch(const tsenor::Params& P, cudaStream_t st) {
+    // a slab (single block column) is cut into panels of vertically stacked blocks
+    const bool tall = (P.cols == M) && (P.rows > M);
+    if constexpr (M < 32) {   // a 32 x 32 block takes a whole warp in either layout
+        const int policy = g_layout.load(std::memory_order_relaxed);
+        bool fine = (policy == TSENOR_LAYOUT_LATENCY);
+        if (policy == TSENOR_LAYOUT_AUTO) {
+            int64_t npc = 0;
+            fine = panel_count<M, 1>(P, tall, &npc) <= 4LL * sm_count();
+        }
+        if (fine) return launch_layout<M, MODE, 1>(P, tall, st);
+    }
+    return launch_layout<M, MODE, 0>(P, tall, st);
 }
 
 template <int MODE>
@@ -531,5 +571,10 @@ const char* tsenor_strerror(int status) {
 int tsenor_last_cuda_error(void) { return g_last_cuda_error; }
 
 int64_t tsenor_launch_count(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
+
+int tsenor_set_layout(int layout) {
+    if (layout < TSENOR_LAYOUT_AUTO || layout > TSENOR_LAYOUT_LATENCY) return TSENOR_ERR_ARG;
+    return g_layout.exchange(layout, std::memory_order_relaxed);
+}
 
 }  // extern "C"

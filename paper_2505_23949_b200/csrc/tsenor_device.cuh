@@ -20,25 +20,40 @@ enum : int { DEV_NONFINITE = 1, DEV_UNDERFILLED = 2, DEV_INTERNAL = 4 };
 
 // ---------------------------------------------------------------------------
 // Dykstra register layout.  A block is spread over LPB = PR*PC lanes arranged
-// as PR x PC; each lane keeps an MR x MC sub-tile (4 x 8 floats, 4 x 4 for
-// M = 4).  Row sums are reduced over the PC lanes that share rows, column
-// sums over the PR lanes that share columns.
+// as PR x PC; each lane keeps an MR x MC sub-tile.  Row sums are reduced over
+// the PC lanes that share rows, column sums over the PR lanes that share
+// columns.  Two layouts per block size:
+//   V = 0  throughput: 4 x 8 sub-tiles (4 x 4 for M = 4), the fewest exchanges per
+//          element; used whenever the matrix has enough blocks to fill the GPU;
+//   V = 1  latency (M < 32): a block over M lanes (the most the exchange scheme allows:
+//          every lane must end up owning one row sum and one column sum), i.e. the
+//          shortest chain of dependent work per iteration and 2-4 times as many
+//          warps for the same matrix; used for matrices too small to fill the GPU.
+//          (Butterfly all-reduces in place of reduce-scatter + all-gather halve the
+//          exchange hops but measured no faster: the chain is then bound by the two
+//          reciprocals and the arithmetic between the hops.)
 // ---------------------------------------------------------------------------
-template <int M> struct Tile;
-template <> struct Tile<32> { static constexpr int PR = 8, PC = 4, MR = 4, MC = 8; };
-template <> struct Tile<16> { static constexpr int PR = 4, PC = 2, MR = 4, MC = 8; };
-template <> struct Tile<8>  { static constexpr int PR = 2, PC = 1, MR = 4, MC = 8; };
-template <> struct Tile<4>  { static constexpr int PR = 1, PC = 1, MR = 4, MC = 4; };
+template <int M, int V> struct Tile;
+template <> struct Tile<32, 0> { static constexpr int PR = 8, PC = 4, MR = 4, MC = 8; };
+template <> struct Tile<16, 0> { static constexpr int PR = 4, PC = 2, MR = 4, MC = 8; };
+template <> struct Tile<8, 0>  { static constexpr int PR = 2, PC = 1, MR = 4, MC = 8; };
+template <> struct Tile<4, 0>  { static constexpr int PR = 1, PC = 1, MR = 4, MC = 4; };
+template <> struct Tile<16, 1> { static constexpr int PR = 4, PC = 4, MR = 4, MC = 4; };
+template <> struct Tile<8, 1>  { static constexpr int PR = 4, PC = 2, MR = 2, MC = 4; };
+template <> struct Tile<4, 1>  { static constexpr int PR = 2, PC = 2, MR = 2, MC = 2; };
 
-template <int M> struct Geom {
-    using T = Tile<M>;
+template <int M_, int V_> struct Geom {
+    static constexpr int M = M_, V = V_;
+    using T = Tile<M, V>;
     static constexpr int LPB = T::PR * T::PC;        // lanes per block (Dykstra)
     static constexpr int BPW = 32 / LPB;             // blocks per warp
     static constexpr int PANEL = WARPS * BPW * M;    // panel width in columns
     static constexpr int WS = PANEL + 1;             // shared row stride (floats)
     static constexpr int GPW = 32 / M;               // rounding groups per warp
-    static constexpr int PASSES = BPW / GPW;         // rounding passes per warp
+    static constexpr int PASSES = (BPW + GPW - 1) / GPW;   // rounding passes per warp
     static constexpr int WORDS = PANEL / 32;         // mask words per panel row
+    static_assert(T::MR >= T::PC && T::MC >= T::PR && T::MC % 2 == 0 && (T::MR * T::MC) % 4 == 0, "tile shape");
+    static_assert(T::PR * T::MR == M && T::PC * T::MC == M, "tile covers the block");
 };
 
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -168,11 +183,12 @@ __device__ __forceinline__ bool out_of_window(float p) {
 // (fp32 min) and the FMA pipe are loaded at that block size (measured).
 template <int M> struct UseSat { static constexpr bool value = (M >= 16); };
 
-template <int M>
-__device__ __forceinline__ void dykstra_step(float2 (&V)[Tile<M>::MR][Tile<M>::MC / 2], float (&rs)[Tile<M>::MR],
-                                             float (&Pr)[Tile<M>::MR / Tile<M>::PC],
-                                             float (&Pc)[Tile<M>::MC / Tile<M>::PR], float Nf, float invN) {
-    using T = Tile<M>;
+template <class G>
+__device__ __forceinline__ void dykstra_step(float2 (&V)[G::T::MR][G::T::MC / 2], float (&rs)[G::T::MR],
+                                             float (&Pr)[G::T::MR / G::T::PC],
+                                             float (&Pc)[G::T::MC / G::T::PR], float Nf, float invN) {
+    using T = typename G::T;
+    constexpr int M = G::M;
     constexpr int MR = T::MR, MC = T::MC, PR = T::PR, PC = T::PC;
     constexpr int RO = MR / PC, CO = MC / PR, MP = MC / 2;
     constexpr bool SAT = UseSat<M>::value;
@@ -222,22 +238,23 @@ __device__ __forceinline__ void dykstra_step(float2 (&V)[Tile<M>::MR][Tile<M>::M
     }
 }
 
-template <int M>
-__device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>::MC], float* stash, int lane,
+template <class G>
+__device__ __forceinline__ void dykstra_iterate(float (&t)[G::T::MR][G::T::MC], float* stash, int lane,
                                                 float Nf, float log2N, int iters) {
-    using T = Tile<M>;
+    using T = typename G::T;
     constexpr int MR = T::MR, MC = T::MC, PR = T::PR, PC = T::PC;
     constexpr int RO = MR / PC, CO = MC / PR;  // lines whose sums this lane finishes
     constexpr int MP = MC / 2, NQ = MR * MC / 4;
-    float F[MR], G[MC];
+    float F[MR], Gc[MC];
     Comp Fo[RO], Go[CO];
     float Pr[RO], Pc[CO];                      // products of rho / kap since the last rebuild
     if (iters <= 0) return;
     float4* const st4 = reinterpret_cast<float4*>(stash) + lane;
 #pragma unroll
-    for (int q = 0; q < NQ; ++q) {
-        const int a = (4 * q) / MC, b = (4 * q) % MC;
-        st4[q * 32] = make_float4(t[a][b], t[a][b + 1], t[a][b + 2], t[a][b + 3]);
+    for (int q = 0; q < NQ; ++q) {   // sub-tile in row-major order, four elements per slot
+        const int e = 4 * q;
+        st4[q * 32] = make_float4(t[e / MC][e % MC], t[(e + 1) / MC][(e + 1) % MC], t[(e + 2) / MC][(e + 2) % MC],
+                                  t[(e + 3) / MC][(e + 3) % MC]);
     }
     {   // iteration 0, log domain
         float rp[MR];
@@ -294,19 +311,19 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>:
 #pragma unroll
         for (int k = 0; k < RO; ++k) { Fo[k].add(lg2_approx(Pr[k])); Pr[k] = 1.0f; F[k] = Fo[k].hi; }
 #pragma unroll
-        for (int k = 0; k < CO; ++k) { Go[k].add(lg2_approx(Pc[k])); Pc[k] = 1.0f; G[k] = Go[k].hi; }
+        for (int k = 0; k < CO; ++k) { Go[k].add(lg2_approx(Pc[k])); Pc[k] = 1.0f; Gc[k] = Go[k].hi; }
         all_gather<MR, PC>(F, 1);
-        all_gather<MC, PR>(G, PC);
+        all_gather<MC, PR>(Gc, PC);
 #pragma unroll
-        for (int q = 0; q < NQ; ++q) {
-            const int a = (4 * q) / MC, b = ((4 * q) % MC) / 2;
+        for (int q = 0; q < NQ; ++q) {   // pairs never straddle a row (MC is even)
+            const int a0 = (4 * q) / MC, b0 = (4 * q) % MC, a1 = (4 * q + 2) / MC, b1 = (4 * q + 2) % MC;
             const float4 v = st4[q * 32];
-            const float2 Fa = make_float2(F[a], F[a]);
-            const float2 x0 = __fadd2_rn(__fadd2_rn(make_float2(v.x, v.y), Fa), make_float2(G[2 * b], G[2 * b + 1]));
-            const float2 x1 =
-                __fadd2_rn(__fadd2_rn(make_float2(v.z, v.w), Fa), make_float2(G[2 * b + 2], G[2 * b + 3]));
-            V[a][b] = make_float2(ex2_approx(x0.x), ex2_approx(x0.y));
-            V[a][b + 1] = make_float2(ex2_approx(x1.x), ex2_approx(x1.y));
+            const float2 x0 = __fadd2_rn(__fadd2_rn(make_float2(v.x, v.y), make_float2(F[a0], F[a0])),
+                                         make_float2(Gc[b0], Gc[b0 + 1]));
+            const float2 x1 = __fadd2_rn(__fadd2_rn(make_float2(v.z, v.w), make_float2(F[a1], F[a1])),
+                                         make_float2(Gc[b1], Gc[b1 + 1]));
+            V[a0][b0 / 2] = make_float2(ex2_approx(x0.x), ex2_approx(x0.y));
+            V[a1][b1 / 2] = make_float2(ex2_approx(x1.x), ex2_approx(x1.y));
         }
 #pragma unroll
         for (int a = 0; a < MR; ++a) rs[a] = 1.0f;     // R_i = 1 (and 1/R_i = 1)
@@ -315,7 +332,7 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>:
 #pragma unroll 1
         while (!wide && it + CHECK <= run_end) {
 #pragma unroll
-            for (int u = 0; u < CHECK; ++u) dykstra_step<M>(V, rs, Pr, Pc, Nf, invN);
+            for (int u = 0; u < CHECK; ++u) dykstra_step<G>(V, rs, Pr, Pc, Nf, invN);
             it += CHECK;
             // exponent field in [127-16, 127+16] <=> product in [2^-16, 2^17).  A product that
             // is inf or NaN (exponent field 255: a block poisoned by a non-finite score) does
@@ -329,24 +346,24 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[Tile<M>::MR][Tile<M>:
         }
         if (!wide) {   // fewer than CHECK iterations left (end of the last run only)
 #pragma unroll 1
-            for (; it < run_end; ++it) dykstra_step<M>(V, rs, Pr, Pc, Nf, invN);
+            for (; it < run_end; ++it) dykstra_step<G>(V, rs, Pr, Pc, Nf, invN);
         }
     }
     // final potentials and t = t0 + F + G
 #pragma unroll
     for (int k = 0; k < RO; ++k) { Fo[k].add(lg2_approx(Pr[k])); F[k] = Fo[k].hi; }
 #pragma unroll
-    for (int k = 0; k < CO; ++k) { Go[k].add(lg2_approx(Pc[k])); G[k] = Go[k].hi; }
+    for (int k = 0; k < CO; ++k) { Go[k].add(lg2_approx(Pc[k])); Gc[k] = Go[k].hi; }
     all_gather<MR, PC>(F, 1);
-    all_gather<MC, PR>(G, PC);
+    all_gather<MC, PR>(Gc, PC);
 #pragma unroll
     for (int q = 0; q < NQ; ++q) {
-        const int a = (4 * q) / MC, b = (4 * q) % MC;
+        const int e = 4 * q;
         const float4 v = st4[q * 32];
-        t[a][b] = (v.x + F[a]) + G[b];
-        t[a][b + 1] = (v.y + F[a]) + G[b + 1];
-        t[a][b + 2] = (v.z + F[a]) + G[b + 2];
-        t[a][b + 3] = (v.w + F[a]) + G[b + 3];
+        t[e / MC][e % MC] = (v.x + F[e / MC]) + Gc[e % MC];
+        t[(e + 1) / MC][(e + 1) % MC] = (v.y + F[(e + 1) / MC]) + Gc[(e + 1) % MC];
+        t[(e + 2) / MC][(e + 2) % MC] = (v.z + F[(e + 2) / MC]) + Gc[(e + 2) % MC];
+        t[(e + 3) / MC][(e + 3) % MC] = (v.w + F[(e + 3) / MC]) + Gc[(e + 3) % MC];
     }
 }
 
@@ -437,10 +454,10 @@ template <int M> struct PanelMap {
 // loads when the addresses allow it.  Return non-zero if a non-finite value
 // was seen by this thread.
 // ---------------------------------------------------------------------------
-template <int M>
-__device__ __forceinline__ int load_score_panel(const ScoreSrc& S, const PanelMap<M>& pm,
+template <class G>
+__device__ __forceinline__ int load_score_panel(const ScoreSrc& S, const PanelMap<G::M>& pm,
                                                 float* __restrict__ dst) {
-    using G = Geom<M>;
+    constexpr int M = G::M;
     constexpr int V = G::PANEL / 4;
     int bad = 0;
     for (int idx = threadIdx.x; idx < M * V; idx += WARPS * 32) {
@@ -454,10 +471,10 @@ __device__ __forceinline__ int load_score_panel(const ScoreSrc& S, const PanelMa
     return bad;
 }
 
-template <int M>
-__device__ __forceinline__ int load_key_panel(const float* __restrict__ src, int64_t ld, const PanelMap<M>& pm,
+template <class G>
+__device__ __forceinline__ int load_key_panel(const float* __restrict__ src, int64_t ld, const PanelMap<G::M>& pm,
                                               bool vec_ok, float* __restrict__ dst) {
-    using G = Geom<M>;
+    constexpr int M = G::M;
     constexpr int V = G::PANEL / 4;
     int bad = 0;
     for (int idx = threadIdx.x; idx < M * V; idx += WARPS * 32) {
@@ -597,10 +614,10 @@ template <int M> __device__ __forceinline__ unsigned transpose_bits(unsigned x, 
 //   lane's column-prefix table when it does not fit in the key cells (M = 32).
 //   tb: the group's scratch; active: group has a block.
 // Returns this lane's row of the mask (M bits).  flags accumulates DEV_* bits.
-template <int M>
-__device__ __forceinline__ unsigned round_block(float* ks, const float* ws, unsigned* cpre, RoundScratch<M>& tb,
+template <class G>
+__device__ __forceinline__ unsigned round_block(float* ks, const float* ws, unsigned* cpre, RoundScratch<G::M>& tb,
                                                 int lane, bool active, int N, int ls_steps, int& flags) {
-    using G = Geom<M>;
+    constexpr int M = G::M;
     constexpr int WS = G::WS;
     constexpr unsigned GM = (M == 32) ? 0xffffffffu : ((1u << (M & 31)) - 1u);
     const int i = lane % M;            // my row, and my column
@@ -732,32 +749,32 @@ struct Params {
     int vec_keys;
 };
 
-template <int M, int MODE> struct SmemLayout {
-    using G = Geom<M>;
+template <class G, int MODE> struct SmemLayout {
+    static constexpr int M = G::M;
     float w[M * G::WS];
     float k[M * G::WS];
     RoundScratch<M> tb[WARPS * G::GPW];
     unsigned int bits[M * G::WORDS];
     unsigned int cpre[(M == 32) ? WARPS * 32 * CPRE_STRIDE : 1];   // column-prefix tables (M = 32)
 };
-template <int M> struct SmemLayout<M, 1> {   // Algorithm 1 alone: score panel and the t0 stash
-    using G = Geom<M>;
+template <class G> struct SmemLayout<G, 1> {   // Algorithm 1 alone: score panel and the t0 stash
+    static constexpr int M = G::M;
     float w[M * G::WS];
-    float k[WARPS * 32 * Tile<M>::MR * Tile<M>::MC];
+    float k[WARPS * 32 * G::T::MR * G::T::MC];
     RoundScratch<M> tb[1];
     unsigned int bits[1];
     unsigned int cpre[1];
 };
 // Resident CTAs per SM the register allocation aims for.
-template <int M> struct MinBlocks { static constexpr int value = (M == 4) ? 5 : 4; };
+template <int M, int V> struct MinBlocks { static constexpr int value = (V == 1) ? 4 : (M == 4) ? 5 : 4; };
 
-template <int M, int MODE>
-__global__ void __launch_bounds__(WARPS * 32, MinBlocks<M>::value) tsenor_kernel(const Params P) {
-    using G = Geom<M>;
-    using T = Tile<M>;
+template <int M, int MODE, int V>
+__global__ void __launch_bounds__(WARPS * 32, MinBlocks<M, V>::value) tsenor_kernel(const Params P) {
+    using G = Geom<M, V>;
+    using T = typename G::T;
     constexpr int MR = T::MR, MC = T::MC, PR = T::PR, PC = T::PC;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    SmemLayout<M, MODE>& sm = *reinterpret_cast<SmemLayout<M, MODE>*>(smem_raw);
+    SmemLayout<G, MODE>& sm = *reinterpret_cast<SmemLayout<G, MODE>*>(smem_raw);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t panel = blockIdx.x;
@@ -778,9 +795,9 @@ __global__ void __launch_bounds__(WARPS * 32, MinBlocks<M>::value) tsenor_kernel
     int flags = 0;
 
     // ---- block loader
-    if (load_score_panel<M>(P.src, pm, sm.w)) flags |= DEV_NONFINITE;
+    if (load_score_panel<G>(P.src, pm, sm.w)) flags |= DEV_NONFINITE;
     if (MODE == 2)
-        if (load_key_panel<M>(P.keys, P.ld_keys, pm, P.vec_keys != 0, sm.k)) flags |= DEV_NONFINITE;
+        if (load_key_panel<G>(P.keys, P.ld_keys, pm, P.vec_keys != 0, sm.k)) flags |= DEV_NONFINITE;
     if (MODE != 1)
         for (int idx = threadIdx.x; idx < M * G::WORDS; idx += WARPS * 32) sm.bits[idx] = 0u;
     __syncthreads();
@@ -831,7 +848,7 @@ __global__ void __launch_bounds__(WARPS * 32, MinBlocks<M>::value) tsenor_kernel
 #pragma unroll
                 for (int b = 0; b < MC; ++b) t[a][b] = fmaf(t[a][b], c_lo, fmaf(t[a][b], c_hi, -sh));
             }
-            dykstra_iterate<M>(t, sm.k + warp * (32 * MR * MC), lane, P.Nf, P.log2N, P.iters);
+            dykstra_iterate<G>(t, sm.k + warp * (32 * MR * MC), lane, P.Nf, P.log2N, P.iters);
 #pragma unroll
             for (int a = 0; a < MR; ++a)
 #pragma unroll
@@ -871,9 +888,9 @@ __global__ void __launch_bounds__(WARPS * 32, MinBlocks<M>::value) tsenor_kernel
 #pragma unroll 1
         for (int pass = 0; pass < G::PASSES; ++pass) {
             const int blk = warp * G::BPW + pass * G::GPW + grp;
-            const bool active = blk * M < valid_cols;
+            const bool active = (pass * G::GPW + grp < G::BPW) && blk * M < valid_cols;
             const unsigned row_bits =
-                round_block<M>(sm.k + blk * M, sm.w + blk * M, sm.cpre + (warp * 32 + lane) * CPRE_STRIDE, tb, lane,
+                round_block<G>(sm.k + blk * M, sm.w + blk * M, sm.cpre + (warp * 32 + lane) * CPRE_STRIDE, tb, lane,
                                active, P.N, P.ls_steps, flags);
             if (active) {
                 const int off = blk * M;

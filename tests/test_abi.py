@@ -60,3 +60,22 @@ def test_binding_refuses_cpu_tensors(lib):
     import torch
     with pytest.raises(TypeError):
         ts.solve(torch.zeros(8, 8), 2, 4, 1.0)
+
+
+def test_layout_setting_is_validated_and_returns_the_previous_value(lib):
+    assert lib.tsenor_set_layout(7) == ts.ERR_ARG and lib.tsenor_set_layout(-1) == ts.ERR_ARG
+    assert ts.set_layout(ts.LAYOUT_LATENCY) == ts.LAYOUT_AUTO
+    assert ts.set_layout(ts.LAYOUT_THROUGHPUT) == ts.LAYOUT_LATENCY
+    assert ts.set_layout(ts.LAYOUT_AUTO) == ts.LAYOUT_THROUGHPUT
+    with pytest.raises(ts.TsenorError):
+        ts.set_layout(3)
+
+
+def test_output_tensor_checks_raise_before_anything_reaches_the_library():
+    """The binding rejects outputs of the wrong kind on the host (no CUDA call is made)."""
+    import torch
+    cpu = torch.zeros(8, 1, dtype=torch.int32)
+    for bad, kw in [(cpu, dict(dtype=torch.int32, device="cuda:0")),]:
+        with pytest.raises(TypeError):
+            ts._out(bad, "mask_out", kw["dtype"], kw["device"])
+    assert ts._out(None, "status", torch.int32, "cuda:0") is None

@@ -8,6 +8,15 @@ import oracle
 from paper_2505_23949_b200 import binding as ts
 
 pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(autouse=True, params=["throughput", "latency"])
+def _both_register_layouts(request):
+    """Every case runs under both register layouts of the Dykstra stage (these matrices are
+    small, so the automatic choice alone would never exercise the throughput layout)."""
+    ts.set_layout(ts.LAYOUT_THROUGHPUT if request.param == "throughput" else ts.LAYOUT_LATENCY)
+    yield
+    ts.set_layout(ts.LAYOUT_AUTO)
 DEV = "cuda:0"
 
 

@@ -12,6 +12,15 @@ from paper_2505_23949_b200 import synth
 
 pytestmark = pytest.mark.gpu
 
+
+@pytest.fixture(autouse=True, params=["throughput", "latency"])
+def _both_register_layouts(request):
+    """Every case runs under both register layouts of the Dykstra stage (these matrices are
+    small, so the automatic choice alone would never exercise the throughput layout)."""
+    ts.set_layout(ts.LAYOUT_THROUGHPUT if request.param == "throughput" else ts.LAYOUT_LATENCY)
+    yield
+    ts.set_layout(ts.LAYOUT_AUTO)
+
 PLAN_TOL = 1e-4
 OBJ_RTOL = 1e-4
 DEV = "cuda:0"
@@ -266,3 +275,19 @@ def test_degenerate_score_matrices(M, N):
     assert np.array_equal(_bits(ts.solve(_dev(const), N, M, 200.0 / 0.37, 300)),
                           oracle.solve(const, N, M, 200.0 / 0.37, 300))
     assert np.array_equal(_bits(ts.solve(_dev(zero), N, M, 1.0, 300)), oracle.solve(zero, N, M, 1.0, 300))
+
+
+def test_binding_rejects_outputs_of_the_wrong_shape_dtype_or_layout():
+    W = _dev(_scores("gauss", 16, 64, 3))
+    with pytest.raises(ValueError):
+        ts.solve(W, 4, 8, 1.0, 1, mask_out=torch.empty((16, 1), dtype=torch.int32, device=DEV))
+    with pytest.raises(TypeError):
+        ts.solve(W, 4, 8, 1.0, 1, mask_out=torch.empty((16, 2), dtype=torch.int64, device=DEV))
+    with pytest.raises(ValueError):
+        ts.solve(W, 4, 8, 1.0, 1, mask_out=torch.empty((16, 4), dtype=torch.int32, device=DEV)[:, ::2])
+    with pytest.raises(TypeError):
+        ts.solve(W, 4, 8, 1.0, 1, status=torch.zeros(1, dtype=torch.int64, device=DEV))
+    with pytest.raises(ValueError):
+        ts.dykstra(W, 4, 8, 1.0, 1, plan_out=torch.empty((16, 32), device=DEV))
+    with pytest.raises(ValueError):
+        ts.objective(W, torch.empty((8, 2), dtype=torch.int32, device=DEV))
