@@ -145,14 +145,16 @@ def aggregate_rate(units_per_rank_per_step, steps, world, elapsed_ms):
 
 
 WORKLOADS = ("config4", "config0", "config1", "config2", "config3", "config5", "admm", "admm_small", "wanda",
-             "sparsegpt")
+             "sparsegpt", "config4_earlyexit")
+EARLY_EXIT_EPS = 1e-3
 
 
 class Job:
     """One tsenor call of a step: host arrays, how to build its score source, N:M."""
 
-    def __init__(self, name, N, M, arrays, kind="abs", scalar=0.0):
+    def __init__(self, name, N, M, arrays, kind="abs", scalar=0.0, ee_eps=0.0):
         self.name, self.N, self.M, self.arrays, self.kind, self.scalar = name, N, M, arrays, kind, scalar
+        self.ee_eps = ee_eps
         self.rows, self.cols = arrays["w"].shape
         self.blocks = (self.rows // M) * (self.cols // M)
         self.score_bytes = self.rows * self.cols * 4          # fp32 scores the mask is computed from
@@ -164,6 +166,9 @@ def make_jobs(workload, index):
     rng = np.random.Generator(np.random.PCG64(977 + index))
     if workload == "config4":
         return [Job(w.name, w.N, w.M, {"w": w.scores})
+                for w in (synth.config(4, index=index, part="up"), synth.config(4, index=index, part="down"))]
+    if workload == "config4_earlyexit":   # the headline matrices in the stopping-test mode (non-parity)
+        return [Job(w.name, w.N, w.M, {"w": w.scores}, kind="abs_ee", ee_eps=EARLY_EXIT_EPS)
                 for w in (synth.config(4, index=index, part="up"), synth.config(4, index=index, part="down"))]
     if workload == "config1":     # 16 different matrices per step: a single 50 us launch between two
         jobs = []                 # event records would time the host's launch path, not the kernel
@@ -224,6 +229,9 @@ WORKLOAD_TEXT = {
     "admm_small": "ADMM D-update on 1024x1024 layers (latency case: 4096 blocks per matrix): scores (W+V/rho)^2 "
                   "computed in the loader, 8:16, then the keep-previous-mask safeguard; 8 different layers per step, "
                   "launches back to back",
+    "config4_earlyexit": "config 4 matrices in the stopping-test mode of Algorithm 1 (NOT the parity contract): a "
+                         "block stops once its marginal violation is below 1e-3 (tested every 4 iterations, at most "
+                         "300); roofline figures count the iterations actually run",
     "wanda": "Wanda scores |W_ij| a_j computed in the loader from bf16 W (4096x4096) and fp32 a_j, 8:16",
     "sparsegpt": "SparseGPT column groups: eight 14336x32 slabs solved one after the other (latency case: 448 "
                  "blocks per call), scores |W_ij / d_j| computed in the loader, 16:32",
@@ -271,7 +279,10 @@ def time_oracle(job, blocks_wanted, want_masks=False):
     sample, nblk, mx = oracle_sample(job, blocks_wanted)
     tau = synth.default_tau(mx)
     t0 = time.perf_counter()
-    bits = oracle.solve(sample, job.N, job.M, tau, T_ITERS, LS_STEPS)
+    if job.ee_eps > 0:
+        bits, _ = oracle.solve_earlyexit(sample, job.N, job.M, tau, T_ITERS, job.ee_eps, 4, LS_STEPS)
+    else:
+        bits = oracle.solve(sample, job.N, job.M, tau, T_ITERS, LS_STEPS)
     dt = time.perf_counter() - t0
     if want_masks:
         return nblk / dt, nblk, dt, oracle.num_threads(), sample, bits
@@ -360,6 +371,7 @@ def run_cuda(args, rank, world, local_rank):
             self.mask = ts.new_mask(job.rows, job.cols, dev)
             self.prev = ts.new_mask(job.rows, job.cols, dev) if job.kind == "admm" else None
             self.obj2 = torch.zeros(2, dtype=torch.float64, device=dev)
+            self.iters_run = torch.zeros(1, dtype=torch.int64, device=dev)   # stopping-test mode only
             self.host_mask = torch.empty(self.mask.shape, dtype=self.mask.dtype).pin_memory()
             self.src_res = self.source(self.res)
             self.tau = synth.default_tau(float(ts.scores_max(self.src_res).item()))
@@ -373,6 +385,8 @@ def run_cuda(args, rank, world, local_rank):
                 return ts.Scores(ts.SCORES_COLMUL, t["w"].view(torch.bfloat16), colvec=t["a"])
             if j.kind == "coldiv":
                 return ts.Scores(ts.SCORES_COLDIV, t["w"], colvec=t["d"])
+            if j.kind == "abs_ee":
+                return ts.Scores(ts.SCORES_ABS, t["w"], early_exit_eps=j.ee_eps, iters_out=self.iters_run)
             return ts.Scores(ts.SCORES_ABS, t["w"])
 
         def solve(self, tensors, src, stream=None):
@@ -422,6 +436,8 @@ def run_cuda(args, rank, world, local_rank):
         barrier()
         cfg["launch"] = "one step captured in a CUDA graph and replayed"
 
+    for d in djobs:
+        d.iters_run.zero_()
     # ---- timed region: inputs resident in HBM
     sampler = ClockSampler(local_rank) if rank == 0 else None
     n0 = ts.launch_count()
@@ -453,6 +469,9 @@ def run_cuda(args, rank, world, local_rank):
     else:
         total_ms = t_begin.elapsed_time(t_end)
     total_ms = max_over_ranks(total_ms, world, dev)
+    # iterations per block actually run (T_ITERS unless the stopping-test mode is on)
+    t_eff = [float(d.iters_run.item()) / (d.job.blocks * args.steps) if d.job.ee_eps > 0 else float(T_ITERS)
+             for d in djobs]
     flags = int(status.item())
     bad = sum(int(ts.check(d.result(), d.job.rows, d.job.cols, d.job.N, d.job.M).item()) for d in djobs)
 
@@ -537,10 +556,10 @@ def run_cuda(args, rank, world, local_rank):
         xu_peak = SM_COUNT * XU_PER_CLK_PER_SM * clk_hz
         # dominant kernel = the solve launches; achieved = algorithmic lane-ops / their CUDA-event time
         solve_s = sum(sum(row) for row in launch_ms) / 1e3
-        ops = args.steps * sum(fp32_lane_ops_per_block(j.M, T_ITERS) * j.blocks for j in jobs)
+        ops = args.steps * sum(fp32_lane_ops_per_block(j.M, te) * j.blocks for j, te in zip(jobs, t_eff))
         achieved = ops / solve_s
-        t_sfu_one = args.steps * sum(xu_ops_per_block_one_exp(j.M, T_ITERS) * j.blocks for j in jobs) / xu_peak
-        t_sfu_lit = args.steps * sum(xu_ops_per_block_literal(j.M, T_ITERS) * j.blocks for j in jobs) / xu_peak
+        t_sfu_one = args.steps * sum(xu_ops_per_block_one_exp(j.M, te) * j.blocks for j, te in zip(jobs, t_eff)) / xu_peak
+        t_sfu_lit = args.steps * sum(xu_ops_per_block_literal(j.M, te) * j.blocks for j, te in zip(jobs, t_eff)) / xu_peak
         alg_bytes = sum(j.h2d_bytes + j.rows * ((j.cols + 31) // 32) * 4 for j in jobs)
         out = {
             "metric": "blocks_per_s", "value": value, "unit": "blocks/s", "n_gpus": world,
@@ -549,6 +568,7 @@ def run_cuda(args, rank, world, local_rank):
             "data": "synthetic", "config": cfg,
             "gb_scores_per_s": world * bytes_per_step * args.steps / sec / 1e9,
             "infeasible_blocks": bad, "dev_status": flags,
+            "mean_iterations_per_block": sum(te * j.blocks for j, te in zip(jobs, t_eff)) / blocks_per_step,
             "clocks": clocks,
             "e2e": {"value": aggregate_rate(blocks_per_step, args.steps, world, e2e_ms), "unit": "blocks/s",
                     "h2d_bytes_per_step": h2d_per_step,
@@ -579,7 +599,7 @@ def run_cuda(args, rank, world, local_rank):
             },
         }
         # spread of the fraction over the timed steps (each step = all launches of the step)
-        step_frac = sorted(sum(fp32_lane_ops_per_block(j.M, T_ITERS) * j.blocks for j in jobs) /
+        step_frac = sorted(sum(fp32_lane_ops_per_block(j.M, te) * j.blocks for j, te in zip(jobs, t_eff)) /
                            (sum(row) / 1e3) / fp32_peak for row in launch_ms)
         out["roofline"]["frac_median"] = statistics.median(step_frac)
         out["roofline"]["frac_min"], out["roofline"]["frac_max"] = step_frac[0], step_frac[-1]

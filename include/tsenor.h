@@ -164,6 +164,18 @@ typedef struct tsenor_scores {
                             block) instead of tau, i.e. the parameter rule of
                             Appendix B.1 applied block by block (pass tau = 200 for
                             "entropy weight 0.005 max|W|"); an all-zero block gets 0  */
+    float early_exit_eps; /* > 0: NON-PARITY performance mode.  Algorithm 1 names T a
+                            "maximum" iteration count without printing a stopping test;
+                            with this set, a block stops before `iters` once the violation
+                            of its marginal constraints, max(max_i |row sum - N|, max_j
+                            |column sum after the row step - N|), seen by an iteration is
+                            below this value.  The test is made at iterations 5, 9, 13, ...
+                            and a warp stops when all the blocks it holds pass (at M = 32
+                            a warp holds one block).  0: fixed iteration count (the
+                            parity contract).                                          */
+    uint64_t *dev_iters_out; /* optional, with or without early_exit_eps: *dev_iters_out
+                            (device, zeroed by the caller) += iterations run, summed over
+                            all blocks                                                 */
 } tsenor_scores_t;
 
 /* tsenor_solve on the score matrix described by *s (same arguments otherwise). */

@@ -69,6 +69,13 @@ def lib():
         L.oracle_keep_better.restype = i32
         L.oracle_simple_round.argtypes = [_f32p, i64, i64, i64, i32, i32, _u32p]
         L.oracle_simple_round.restype = i32
+        L.oracle_dykstra_block_earlyexit.argtypes = [_f64p, i32, i32, f64, i32, f64, i32, _f64p, _f64p]
+        L.oracle_dykstra_block_earlyexit.restype = i32
+        L.oracle_solve_earlyexit.argtypes = [_f32p, i64, i64, i64, i32, i32, f32, i32, i32, f64, i32, _u32p, _i32p]
+        L.oracle_solve_earlyexit.restype = i32
+        L.oracle_dykstra_earlyexit.argtypes = [_f32p, i64, i64, i64, i32, i32, f32, i32, f64, i32, _f64p, i64, i32,
+                                               _i32p]
+        L.oracle_dykstra_earlyexit.restype = i32
         L.oracle_num_threads.argtypes = []
         L.oracle_num_threads.restype = i32
         _lib = L
@@ -165,6 +172,42 @@ def dykstra(scores, N, M, tau, iters, plan_is_log=False, per_block_tau=False):
     _check(fn(s, rows, cols, cols, int(N), int(M), float(tau),
                                 int(iters), plan, cols, int(bool(plan_is_log))), "dykstra")
     return plan
+
+
+def dykstra_block_earlyexit(w, N, tau, max_iters, eps, check_every=1):
+    """Algorithm 1 on one block with the stopping test (marginal violation below ``eps`` at an
+    iteration t = 1 + k * ``check_every``, k >= 1).  Returns ``(x, q, iterations run)``."""
+    w = np.ascontiguousarray(w, dtype=np.float64)
+    M = w.shape[0]
+    x = np.empty((M, M), np.float64)
+    q = np.empty((M, M), np.float64)
+    ran = lib().oracle_dykstra_block_earlyexit(w, M, int(N), float(tau), int(max_iters), float(eps),
+                                               int(check_every), x, q)
+    return x, q, int(ran)
+
+
+def solve_earlyexit(scores, N, M, tau, max_iters, eps, check_every=1, ls_steps=-1):
+    """The whole method with the stopping test in Algorithm 1.  Returns ``(mask bits, iterations
+    run by every block)``."""
+    s = _f32(scores)
+    rows, cols = s.shape
+    bits = np.zeros((rows, mask_words_per_row(cols)), np.uint32)
+    iters = np.zeros((rows // M) * (cols // M), np.int32)
+    _check(lib().oracle_solve_earlyexit(s, rows, cols, cols, int(N), int(M), float(tau), int(max_iters),
+                                        int(ls_steps), float(eps), int(check_every), bits, iters), "solve_earlyexit")
+    return bits, iters
+
+
+def dykstra_earlyexit(scores, N, M, tau, max_iters, eps, check_every=1, plan_is_log=False):
+    """Algorithm 1 with the stopping test on every tile: ``(fp64 plan, iterations per block)``."""
+    s = _f32(scores)
+    rows, cols = s.shape
+    plan = np.empty((rows, cols), np.float64)
+    iters = np.zeros((rows // M) * (cols // M), np.int32)
+    _check(lib().oracle_dykstra_earlyexit(s, rows, cols, cols, int(N), int(M), float(tau), int(max_iters),
+                                          float(eps), int(check_every), plan, cols, int(bool(plan_is_log)), iters),
+           "dykstra_earlyexit")
+    return plan, iters
 
 
 def _stats_arrays(nblk, want):

@@ -123,6 +123,48 @@ void oracle_dykstra_block(const double *w, int M, int N, double tau, int iters,
     if (extra_steps >= 2) project_cols(x, M, N);
 }
 
+/*
+ * Algorithm 1 with a stopping test.  The paper caps the iteration count ("maximum
+ * iterations T", Algorithm 1; "limit the maximum iterations to T = 300", Appendix B.1)
+ * without printing a test; this variant (not the parity contract, which is the fixed
+ * count above) uses the violation of the two marginal constraints seen by iteration t:
+ *   delta_t = max( max_i |sum_j S(t-1)_ij - N| ,  max_j |sum_i S'_ij - N| ),
+ * S(t-1) the iterate entering iteration t (after the previous clip) and S' the same after
+ * the row step of iteration t.  Iteration t is always completed (column step, clip, dual
+ * update); the loop stops after it when delta_t < eps and t is one of the iterations at
+ * which the test is made: t = 1 + k * check_every, k >= 1.  eps <= 0 never stops early.
+ * Returns the number of iterations run.
+ */
+int oracle_dykstra_block_earlyexit(const double *w, int M, int N, double tau, int max_iters,
+                                   double eps, int check_every, double *x, double *q)
+{
+    for (int e = 0; e < M * M; ++e) {
+        x[e] = tau * fabs(w[e]);
+        q[e] = 0.0;
+    }
+    if (check_every < 1) check_every = 1;
+    int t = 0;
+    while (t < max_iters) {
+        ++t;
+        double delta = 0.0;
+        for (int i = 0; i < M; ++i) {
+            double s = 0.0;
+            for (int j = 0; j < M; ++j) s += exp(x[(size_t)i * M + j]);
+            if (fabs(s - N) > delta) delta = fabs(s - N);
+        }
+        project_rows(x, M, N);
+        for (int j = 0; j < M; ++j) {
+            double s = 0.0;
+            for (int i = 0; i < M; ++i) s += exp(x[(size_t)i * M + j]);
+            if (fabs(s - N) > delta) delta = fabs(s - N);
+        }
+        project_cols(x, M, N);
+        project_cap(x, q, M);
+        if (eps > 0.0 && t > 1 && (t - 1) % check_every == 0 && delta < eps) break;
+    }
+    return t;
+}
+
 /* ------------------------------------------------------------------ */
 /* Algorithm 2                                                         */
 /* ------------------------------------------------------------------ */
@@ -358,7 +400,8 @@ static double tau_of_block(double tau, int per_block, const double *w, int M)
 
 static int dykstra_matrix(const float *scores, int64_t rows, int64_t cols, int64_t ld,
                    int N, int M, float tau, int per_block, int iters, double *plan_out,
-                   int64_t ld_plan, int plan_is_log)
+                   int64_t ld_plan, int plan_is_log, double eps, int check_every,
+                   int32_t *blk_iters)
 {
     if (!scores || !plan_out || !check_shape(rows, cols, N, M) || iters < 0 ||
         N < 1 || N >= M)
@@ -372,7 +415,13 @@ static int dykstra_matrix(const float *scores, int64_t rows, int64_t cols, int64
         for (int64_t b = 0; b < nbr * nbc; ++b) {
             int64_t r0 = (b / nbc) * M, c0 = (b % nbc) * M;
             gather_block_abs(scores, ld, r0, c0, M, w, NULL);
-            oracle_dykstra_block(w, M, N, tau_of_block((double)tau, per_block, w, M), iters, 0, x, q);
+            int ran = iters;
+            if (eps > 0.0)
+                ran = oracle_dykstra_block_earlyexit(w, M, N, tau_of_block((double)tau, per_block, w, M),
+                                                     iters, eps, check_every, x, q);
+            else
+                oracle_dykstra_block(w, M, N, tau_of_block((double)tau, per_block, w, M), iters, 0, x, q);
+            if (blk_iters) blk_iters[b] = ran;
             for (int i = 0; i < M; ++i)
                 for (int j = 0; j < M; ++j)
                     plan_out[(size_t)(r0 + i) * ld_plan + (c0 + j)] =
@@ -476,7 +525,8 @@ int oracle_round(const float *plan_key, int64_t ld_plan, const float *scores,
 static int solve_matrix(const float *scores, int64_t rows, int64_t cols, int64_t ld,
                  int N, int M, float tau, int per_block, int iters, int ls_steps,
                  uint32_t *mask_bits, int32_t *blk_steps, int32_t *blk_nonpos,
-                 double *blk_obj, int64_t *underfilled)
+                 double *blk_obj, int64_t *underfilled, double eps, int check_every,
+                 int32_t *blk_iters)
 {
     if (!scores || !mask_bits || !check_shape(rows, cols, N, M) || iters < 0 ||
         N < 1 || N >= M)
@@ -496,7 +546,13 @@ static int solve_matrix(const float *scores, int64_t rows, int64_t cols, int64_t
             for (int64_t bc = 0; bc < nbc; ++bc) {
                 int64_t r0 = br * M, c0 = bc * M, b = br * nbc + bc;
                 gather_block_abs(scores, ld, r0, c0, M, w, wf);
-                oracle_dykstra_block(w, M, N, tau_of_block((double)tau, per_block, w, M), iters, 0, x, q);
+                int ran = iters;
+                if (eps > 0.0)
+                    ran = oracle_dykstra_block_earlyexit(w, M, N, tau_of_block((double)tau, per_block, w, M),
+                                                         iters, eps, check_every, x, q);
+                else
+                    oracle_dykstra_block(w, M, N, tau_of_block((double)tau, per_block, w, M), iters, 0, x, q);
+                if (blk_iters) blk_iters[b] = ran;
                 int steps, nonpos;
                 double obj;
                 int ok = round_one(x, wf, M, N, ls_steps, S, R, C, &steps,
@@ -522,7 +578,7 @@ int oracle_solve(const float *scores, int64_t rows, int64_t cols, int64_t ld,
                  double *blk_obj, int64_t *underfilled)
 {
     return solve_matrix(scores, rows, cols, ld, N, M, tau, 0, iters, ls_steps, mask_bits,
-                        blk_steps, blk_nonpos, blk_obj, underfilled);
+                        blk_steps, blk_nonpos, blk_obj, underfilled, 0.0, 1, NULL);
 }
 
 /* Per-block variant: block b runs with tau = tau_rel / max|score| of block b. */
@@ -532,21 +588,41 @@ int oracle_solve_blocktau(const float *scores, int64_t rows, int64_t cols, int64
                           double *blk_obj, int64_t *underfilled)
 {
     return solve_matrix(scores, rows, cols, ld, N, M, tau_rel, 1, iters, ls_steps, mask_bits,
-                        blk_steps, blk_nonpos, blk_obj, underfilled);
+                        blk_steps, blk_nonpos, blk_obj, underfilled, 0.0, 1, NULL);
+}
+
+/* The whole method with the stopping test of oracle_dykstra_block_earlyexit in Algorithm 1;
+ * blk_iters (optional) receives the iterations each block ran. */
+int oracle_solve_earlyexit(const float *scores, int64_t rows, int64_t cols, int64_t ld,
+                           int N, int M, float tau, int max_iters, int ls_steps, double eps,
+                           int check_every, uint32_t *mask_bits, int32_t *blk_iters)
+{
+    return solve_matrix(scores, rows, cols, ld, N, M, tau, 0, max_iters, ls_steps, mask_bits,
+                        NULL, NULL, NULL, NULL, eps, check_every, blk_iters);
+}
+
+int oracle_dykstra_earlyexit(const float *scores, int64_t rows, int64_t cols, int64_t ld,
+                             int N, int M, float tau, int max_iters, double eps, int check_every,
+                             double *plan_out, int64_t ld_plan, int plan_is_log, int32_t *blk_iters)
+{
+    return dykstra_matrix(scores, rows, cols, ld, N, M, tau, 0, max_iters, plan_out, ld_plan,
+                          plan_is_log, eps, check_every, blk_iters);
 }
 
 int oracle_dykstra(const float *scores, int64_t rows, int64_t cols, int64_t ld,
                    int N, int M, float tau, int iters, double *plan_out,
                    int64_t ld_plan, int plan_is_log)
 {
-    return dykstra_matrix(scores, rows, cols, ld, N, M, tau, 0, iters, plan_out, ld_plan, plan_is_log);
+    return dykstra_matrix(scores, rows, cols, ld, N, M, tau, 0, iters, plan_out, ld_plan, plan_is_log, 0.0, 1,
+                          NULL);
 }
 
 int oracle_dykstra_blocktau(const float *scores, int64_t rows, int64_t cols, int64_t ld,
                             int N, int M, float tau_rel, int iters, double *plan_out,
                             int64_t ld_plan, int plan_is_log)
 {
-    return dykstra_matrix(scores, rows, cols, ld, N, M, tau_rel, 1, iters, plan_out, ld_plan, plan_is_log);
+    return dykstra_matrix(scores, rows, cols, ld, N, M, tau_rel, 1, iters, plan_out, ld_plan, plan_is_log, 0.0,
+                          1, NULL);
 }
 
 /* Objective of Eq. 1: sum of |score| over the set bits, in fp64. */

@@ -32,7 +32,7 @@ class ScoresDesc(C.Structure):
     """ctypes image of ``tsenor_scores_t`` (a host struct holding device pointers)."""
     _fields_ = [("kind", C.c_int), ("w_is_bf16", C.c_int), ("w", C.c_void_p), ("ld", C.c_int64),
                 ("v", C.c_void_p), ("ld_v", C.c_int64), ("scalar", C.c_float), ("colvec", C.c_void_p),
-                ("per_block_tau", C.c_int)]
+                ("per_block_tau", C.c_int), ("early_exit_eps", C.c_float), ("dev_iters_out", C.c_void_p)]
 
 _lib = None
 
@@ -257,9 +257,13 @@ def max_abs(scores, out=None, stream=None):
 class Scores:
     """A described score matrix (``tsenor_scores_t``): keeps the tensors alive and builds
     the descriptor.  kind: SCORES_ABS |W|, SCORES_ADMM (W + V*scalar)^2, SCORES_COLDIV
-    |W / colvec_j|, SCORES_COLMUL |W| * colvec_j.  W may be float32 or bfloat16."""
+    |W / colvec_j|, SCORES_COLMUL |W| * colvec_j.  W may be float32 or bfloat16.
+    ``early_exit_eps`` > 0 switches the stopping test of Algorithm 1 on (non-parity mode);
+    ``iters_out`` (1-element int64 device tensor, zeroed by the caller) accumulates the
+    iterations run over all blocks."""
 
-    def __init__(self, kind, w, v=None, scalar=0.0, colvec=None, per_block_tau=False):
+    def __init__(self, kind, w, v=None, scalar=0.0, colvec=None, per_block_tau=False, early_exit_eps=0.0,
+                 iters_out=None):
         if not (isinstance(w, torch.Tensor) and w.is_cuda and w.dim() == 2 and w.stride(1) == 1):
             raise TypeError("w must be a 2-D row-major CUDA tensor")
         if w.dtype not in (torch.float32, torch.bfloat16):
@@ -283,6 +287,10 @@ class Scores:
                 raise TypeError("colvec must be a contiguous float32 CUDA vector of length cols on w's device")
             d.colvec = colvec.data_ptr()
         d.per_block_tau = int(bool(per_block_tau))
+        d.early_exit_eps = float(early_exit_eps)
+        self.iters_out = _out(iters_out, "iters_out", torch.int64, w.device, min_numel=1)
+        if iters_out is not None:
+            d.dev_iters_out = iters_out.data_ptr()
         self.desc = d
 
     @property

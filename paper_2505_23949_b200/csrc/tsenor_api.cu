@@ -350,7 +350,21 @@ int trivial_mask(uint32_t* bits, int64_t rows, int64_t cols, bool ones, cudaStre
 
 extern "C" {
 
-static int solve_on(const tsenor::ScoreSrc& src, int per_block_tau, int64_t rows, int64_t cols, int N, int M,
+struct Extras {   // optional settings carried by tsenor_scores_t
+    int per_block_tau = 0;
+    float ee_eps = 0.0f;
+    unsigned long long* iter_sum = nullptr;
+};
+
+static int extras_of(const tsenor_scores_t* s, Extras* x) {
+    x->per_block_tau = s->per_block_tau ? 1 : 0;
+    if (!(s->early_exit_eps >= 0.0f) || !std::isfinite(s->early_exit_eps)) return TSENOR_ERR_ARG;
+    x->ee_eps = s->early_exit_eps;
+    x->iter_sum = reinterpret_cast<unsigned long long*>(s->dev_iters_out);
+    return TSENOR_OK;
+}
+
+static int solve_on(const tsenor::ScoreSrc& src, const Extras& x, int64_t rows, int64_t cols, int N, int M,
                     float tau, int iters, int ls_steps, uint32_t* mask_bits_out, int32_t* dev_status,
                     cudaStream_t st) {
     if (N == 0 || N == M) return trivial_mask(mask_bits_out, rows, cols, N == M, st);
@@ -360,7 +374,8 @@ static int solve_on(const tsenor::ScoreSrc& src, int per_block_tau, int64_t rows
     P.rows = rows; P.cols = cols;
     P.N = N; P.Nf = (float)N; P.log2N = (float)std::log2((double)N);
     set_tau(P, tau);
-    P.per_block_tau = per_block_tau;
+    P.per_block_tau = x.per_block_tau;
+    P.ee_eps = x.ee_eps; P.iter_sum = x.iter_sum;
     P.iters = iters; P.ls_steps = ls_steps;
     P.status = dev_status;
     return dispatch<0>(P, M, st);
@@ -373,8 +388,8 @@ int tsenor_solve(const float* scores, int64_t rows, int64_t cols, int64_t ld, in
     if (iters < 0 || !(tau >= 0.0f) || !std::isfinite(tau)) return TSENOR_ERR_ARG;
     if (rows == 0 || cols == 0) return TSENOR_OK;
     if (!scores || !mask_bits_out) return TSENOR_ERR_NULL;
-    return solve_on(abs_source(scores, ld), 0, rows, cols, N, M, tau, iters, ls_steps, mask_bits_out, dev_status,
-                    (cudaStream_t)stream);
+    return solve_on(abs_source(scores, ld), Extras{}, rows, cols, N, M, tau, iters, ls_steps, mask_bits_out,
+                    dev_status, (cudaStream_t)stream);
 }
 
 int tsenor_solve_scores(const tsenor_scores_t* s, int64_t rows, int64_t cols, int N, int M, float tau, int iters,
@@ -386,7 +401,9 @@ int tsenor_solve_scores(const tsenor_scores_t* s, int64_t rows, int64_t cols, in
     if (int rc = make_source(s, cols, &src)) return rc;
     if (rows == 0 || cols == 0) return TSENOR_OK;
     if (!mask_bits_out) return TSENOR_ERR_NULL;
-    return solve_on(src, s->per_block_tau ? 1 : 0, rows, cols, N, M, tau, iters, ls_steps, mask_bits_out, dev_status,
+    Extras x;
+    if (int rc = extras_of(s, &x)) return rc;
+    return solve_on(src, x, rows, cols, N, M, tau, iters, ls_steps, mask_bits_out, dev_status,
                     (cudaStream_t)stream);
 }
 
@@ -452,7 +469,7 @@ int tsenor_simple_round(const float* plan_key, int64_t ld_plan, int64_t rows, in
     return finish_launch();
 }
 
-static int dykstra_on(const tsenor::ScoreSrc& src, int per_block_tau, int64_t rows, int64_t cols, int N, int M,
+static int dykstra_on(const tsenor::ScoreSrc& src, const Extras& x, int64_t rows, int64_t cols, int N, int M,
                       float tau, int iters, float* plan_out, int64_t ld_plan, int plan_is_log,
                       int32_t* dev_status, cudaStream_t st) {
     tsenor::Params P{};
@@ -461,7 +478,8 @@ static int dykstra_on(const tsenor::ScoreSrc& src, int per_block_tau, int64_t ro
     P.rows = rows; P.cols = cols;
     P.N = N; P.Nf = (float)N; P.log2N = (float)std::log2((double)N);
     set_tau(P, tau);
-    P.per_block_tau = per_block_tau;
+    P.per_block_tau = x.per_block_tau;
+    P.ee_eps = x.ee_eps; P.iter_sum = x.iter_sum;
     P.iters = iters; P.ls_steps = -1;
     P.status = dev_status;
     return dispatch<1>(P, M, st);
@@ -475,7 +493,7 @@ int tsenor_dykstra(const float* scores, int64_t rows, int64_t cols, int64_t ld, 
     if (iters < 0 || !(tau >= 0.0f) || !std::isfinite(tau)) return TSENOR_ERR_ARG;
     if (rows == 0 || cols == 0) return TSENOR_OK;
     if (!scores || !plan_out) return TSENOR_ERR_NULL;
-    return dykstra_on(abs_source(scores, ld), 0, rows, cols, N, M, tau, iters, plan_out, ld_plan, plan_is_log,
+    return dykstra_on(abs_source(scores, ld), Extras{}, rows, cols, N, M, tau, iters, plan_out, ld_plan, plan_is_log,
                       dev_status, (cudaStream_t)stream);
 }
 
@@ -490,7 +508,9 @@ int tsenor_dykstra_scores(const tsenor_scores_t* s, int64_t rows, int64_t cols, 
     if (int rc = make_source(s, cols, &src)) return rc;
     if (rows == 0 || cols == 0) return TSENOR_OK;
     if (!plan_out) return TSENOR_ERR_NULL;
-    return dykstra_on(src, s->per_block_tau ? 1 : 0, rows, cols, N, M, tau, iters, plan_out, ld_plan, plan_is_log,
+    Extras x;
+    if (int rc = extras_of(s, &x)) return rc;
+    return dykstra_on(src, x, rows, cols, N, M, tau, iters, plan_out, ld_plan, plan_is_log,
                       dev_status, (cudaStream_t)stream);
 }
 

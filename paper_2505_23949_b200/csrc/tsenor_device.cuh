@@ -183,10 +183,12 @@ __device__ __forceinline__ bool out_of_window(float p) {
 // (fp32 min) and the FMA pipe are loaded at that block size (measured).
 template <int M> struct UseSat { static constexpr bool value = (M >= 16); };
 
-template <class G>
-__device__ __forceinline__ void dykstra_step(float2 (&V)[G::T::MR][G::T::MC / 2], float (&rs)[G::T::MR],
-                                             float (&Pr)[G::T::MR / G::T::PC],
-                                             float (&Pc)[G::T::MC / G::T::PR], float Nf, float invN) {
+// DELTA: also returns this lane's share of the marginal violation seen by the iteration,
+// max over the lines it owns of |row sum of e - N| and |column sum of e rho - N|.
+template <class G, bool DELTA = false>
+__device__ __forceinline__ float dykstra_step(float2 (&V)[G::T::MR][G::T::MC / 2], float (&rs)[G::T::MR],
+                                              float (&Pr)[G::T::MR / G::T::PC],
+                                              float (&Pc)[G::T::MC / G::T::PR], float Nf, float invN) {
     using T = typename G::T;
     constexpr int M = G::M;
     constexpr int MR = T::MR, MC = T::MC, PR = T::PR, PC = T::PC;
@@ -206,6 +208,11 @@ __device__ __forceinline__ void dykstra_step(float2 (&V)[G::T::MR][G::T::MC / 2]
         rp[a] = s2.x + s2.y;
     }
     reduce_scatter<MR, PC>(rp, 1, OpAdd());
+    float delta = 0.0f;
+    if (DELTA) {   // row sums of e: rp itself (SAT), rp R_i(old) otherwise
+#pragma unroll
+        for (int k = 0; k < RO; ++k) delta = fmaxf(delta, fabsf((SAT ? rp[k] : rp[k] * Pr[k]) - Nf));
+    }
 #pragma unroll
     for (int k = 0; k < RO; ++k) {
         sc[k] = Nf * rcp_approx(rp[k]);          // SAT: rho_i; !SAT: the new R_i
@@ -223,6 +230,10 @@ __device__ __forceinline__ void dykstra_step(float2 (&V)[G::T::MR][G::T::MC / 2]
         cp[2 * b + 1] = c2.y;
     }
     reduce_scatter<MC, PR>(cp, PC, OpAdd());
+    if (DELTA) {
+#pragma unroll
+        for (int k = 0; k < CO; ++k) delta = fmaxf(delta, fabsf(cp[k] - Nf));
+    }
 #pragma unroll
     for (int k = 0; k < CO; ++k) {
         kap[k] = Nf * rcp_approx(cp[k]);
@@ -236,11 +247,15 @@ __device__ __forceinline__ void dykstra_step(float2 (&V)[G::T::MR][G::T::MC / 2]
 #pragma unroll
         for (int b = 0; b < MP; ++b) V[a][b] = __fmul2_rn(V[a][b], make_float2(kap[2 * b], kap[2 * b + 1]));
     }
+    return delta;
 }
 
+// Returns the number of iterations run: iters, or fewer in the stopping-test mode (ee_eps > 0):
+// after every group of CHECK iterations, i.e. at iterations 5, 9, 13, ... of Algorithm 1, the
+// warp stops once the marginal violation of every block it holds is below ee_eps.
 template <class G>
-__device__ __forceinline__ void dykstra_iterate(float (&t)[G::T::MR][G::T::MC], float* stash, int lane,
-                                                float Nf, float log2N, int iters) {
+__device__ __forceinline__ int dykstra_iterate(float (&t)[G::T::MR][G::T::MC], float* stash, int lane,
+                                               float Nf, float log2N, int iters, float ee_eps) {
     using T = typename G::T;
     constexpr int MR = T::MR, MC = T::MC, PR = T::PR, PC = T::PC;
     constexpr int RO = MR / PC, CO = MC / PR;  // lines whose sums this lane finishes
@@ -248,7 +263,7 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[G::T::MR][G::T::MC], 
     float F[MR], Gc[MC];
     Comp Fo[RO], Go[CO];
     float Pr[RO], Pc[CO];                      // products of rho / kap since the last rebuild
-    if (iters <= 0) return;
+    if (iters <= 0) return 0;
     float4* const st4 = reinterpret_cast<float4*>(stash) + lane;
 #pragma unroll
     for (int q = 0; q < NQ; ++q) {   // sub-tile in row-major order, four elements per slot
@@ -331,8 +346,19 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[G::T::MR][G::T::MC], 
         bool wide = false;
 #pragma unroll 1
         while (!wide && it + CHECK <= run_end) {
-#pragma unroll
-            for (int u = 0; u < CHECK; ++u) dykstra_step<G>(V, rs, Pr, Pc, Nf, invN);
+#pragma unroll(G::M == 8 ? 1 : CHECK)   // measured: unrolling the group helps every size but M = 8
+            for (int u = 0; u < CHECK - 1; ++u) dykstra_step<G>(V, rs, Pr, Pc, Nf, invN);
+            if (ee_eps > 0.0f) {
+                const float delta = dykstra_step<G, true>(V, rs, Pr, Pc, Nf, invN);
+                if (__all_sync(FULL, delta < ee_eps)) {   // every block of the warp has converged
+                    it += CHECK;
+                    iters = it;
+                    wide = true;                          // skips the remainder loop as well
+                    break;
+                }
+            } else {
+                dykstra_step<G>(V, rs, Pr, Pc, Nf, invN);
+            }
             it += CHECK;
             // exponent field in [127-16, 127+16] <=> product in [2^-16, 2^17).  A product that
             // is inf or NaN (exponent field 255: a block poisoned by a non-finite score) does
@@ -365,6 +391,7 @@ __device__ __forceinline__ void dykstra_iterate(float (&t)[G::T::MR][G::T::MC], 
         t[(e + 2) / MC][(e + 2) % MC] = (v.z + F[(e + 2) / MC]) + Gc[(e + 2) % MC];
         t[(e + 3) / MC][(e + 3) % MC] = (v.w + F[(e + 3) / MC]) + Gc[(e + 3) % MC];
     }
+    return iters;
 }
 
 // ---------------------------------------------------------------------------
@@ -745,6 +772,8 @@ struct Params {
     float c_hi, c_lo;              // tau * log2(e), split in two floats
     int per_block_tau;             // tau is divided by each block's own largest score
     int iters, ls_steps;
+    float ee_eps;                  // > 0: stopping test of Algorithm 1 (non-parity mode)
+    unsigned long long* iter_sum;  // optional: iterations run, summed over the blocks
     int32_t* status;
     int vec_keys;
 };
@@ -848,7 +877,12 @@ __global__ void __launch_bounds__(WARPS * 32, MinBlocks<M, V>::value) tsenor_ker
 #pragma unroll
                 for (int b = 0; b < MC; ++b) t[a][b] = fmaf(t[a][b], c_lo, fmaf(t[a][b], c_hi, -sh));
             }
-            dykstra_iterate<G>(t, sm.k + warp * (32 * MR * MC), lane, P.Nf, P.log2N, P.iters);
+            const int ran =
+                dykstra_iterate<G>(t, sm.k + warp * (32 * MR * MC), lane, P.Nf, P.log2N, P.iters, P.ee_eps);
+            if (P.iter_sum) {   // one add per warp: iterations x blocks of the warp that exist
+                const int nact = __popc(__ballot_sync(FULL, active && g == 0));
+                if (lane == 0 && nact) atomicAdd(P.iter_sum, (unsigned long long)ran * nact);
+            }
 #pragma unroll
             for (int a = 0; a < MR; ++a)
 #pragma unroll

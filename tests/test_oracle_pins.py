@@ -610,3 +610,42 @@ def test_per_block_tau_is_the_plain_method_block_by_block():
     assert 0 <= gap_pb <= gap_gl
     zero = np.zeros((M, M), np.float32)                    # an all-zero block gets tau = 0
     assert oracle.count_infeasible(oracle.solve(zero, N, M, 200.0, 10, per_block_tau=True), M, M, N, M) == 0
+
+
+def test_stopping_test_variant_of_algorithm1():
+    """The variant of Algorithm 1 with a stopping test: identical to the fixed count when the test
+    is off; the count it returns is the first tested iteration t = 1 + 4k whose marginal violation,
+    recomputed here from the fixed-count oracle's iterates, is below eps; counts fall as eps grows."""
+    rng = np.random.default_rng(61)
+    for M, N, tau in [(4, 2, 30.0), (8, 4, 40.0), (16, 8, 25.0), (32, 16, 12.0), (8, 3, 60.0)]:
+        w = np.abs(rng.standard_normal((M, M)))
+        w /= w.max()
+        x0, q0 = oracle.dykstra_block(w, N, tau, 80)
+        x1, q1, ran = oracle.dykstra_block_earlyexit(w, N, tau, 80, 0.0, 4)
+        assert ran == 80 and np.array_equal(x0, x1) and np.array_equal(q0, q1)
+        prev = 10 ** 9
+        for eps in (1e-6, 1e-4, 1e-2, 0.3):
+            x, q, ran = oracle.dykstra_block_earlyexit(w, N, tau, 400, eps, 4)
+            assert ran <= prev
+            prev = ran
+            first = None
+            for t in range(5, 401, 4):                     # iterations at which the test is made
+                s_in = np.exp(oracle.dykstra_block(w, N, tau, t - 1)[0])              # iterate entering t
+                s_row = np.exp(oracle.dykstra_block(w, N, tau, t - 1, extra_steps=1)[0])  # after its row step
+                delta = max(np.abs(s_in.sum(1) - N).max(), np.abs(s_row.sum(0) - N).max())
+                if delta < eps:
+                    first = t
+                    break
+            assert ran == (first if first is not None else 400), (M, N, eps)
+            xr, qr = oracle.dykstra_block(w, N, tau, ran)      # and it returns that iteration's iterate
+            assert np.array_equal(x, xr) and np.array_equal(q, qr)
+    W = np.abs(rng.standard_normal((32, 48)) * 0.02).astype(np.float32)
+    tau = 15.0 / W.max()
+    bits, iters = oracle.solve_earlyexit(W, 4, 8, tau, 300, 0.0, 4)
+    assert np.array_equal(bits, oracle.solve(W, 4, 8, tau, 300)) and (iters == 300).all()
+    bits, iters = oracle.solve_earlyexit(W, 4, 8, tau, 300, 1e-3, 4)
+    assert iters.max() < 300 and ((iters - 1) % 4 == 0).all()
+    assert oracle.count_infeasible(bits, 32, 48, 4, 8) == 0
+    plan, iters2 = oracle.dykstra_earlyexit(W, 4, 8, tau, 300, 1e-3, 4)
+    assert np.array_equal(iters, iters2)
+    assert np.abs(plan - oracle.dykstra(W, 4, 8, tau, 300)).max() < 5e-3   # stopped close to the fixed point
