@@ -545,50 +545,71 @@ __device__ __forceinline__ unsigned long long sort_word(float key, int idx) {
     return ((unsigned long long)(~u) << 32) | (unsigned)idx;
 }
 
+// The same order packed into one ascending 32-bit word: the high word of sort_word with its
+// five low bits replaced by the index.  Dropping those bits is harmless unless two keys of
+// the line agree in the 27 bits kept ("same bucket"): then their order may depend on the
+// bits dropped, and the caller falls back to the 64-bit words.  Keys that are exactly zero
+// (the capped entries of a plan: up to half of a line) are the one common case of equal
+// keys; each of them gets a bucket of its own, ZERO_BUCKET + index (zeros order among
+// themselves by index), and the positive keys are shifted down by the 32 buckets this takes.
+constexpr unsigned ZERO_BUCKET = 0x03ffffe0u;
+__device__ __forceinline__ unsigned sort_word_packed(float key, unsigned idx) {
+    if (!(key == key)) key = __int_as_float(0xff800000);
+    key += 0.0f;
+    const unsigned b = __float_as_uint(key);
+    unsigned hi;
+    if (b & 0x80000000u) hi = b;                               // negative: larger magnitude later
+    else if (b == 0u) hi = (ZERO_BUCKET + idx) << 5;
+    else hi = 0x7fffffffu - b - (32u * 32u + 31u);             // positive: larger first, all before the zeros
+    return (hi & ~31u) | idx;
+}
+
 // Batcher's odd-even merge sort as a fully unrolled network (191 compare-exchanges for 32
 // keys, 63 for 16, 19 for 8, 5 for 4), ascending.  Indices are template constants so that the
-// keys stay in registers.
+// keys stay in registers.  A compare-exchange costs two instructions on 32-bit words (min,
+// max) and six on 64-bit words.
 template <int I, int J, int M> __device__ __forceinline__ void cmp_swap(unsigned long long (&v)[M]) {
     const unsigned long long a = v[I], b = v[J];
     const bool sw = a > b;
     v[I] = sw ? b : a;
     v[J] = sw ? a : b;
 }
-template <int LO, int N, int R, int I, int M> __device__ __forceinline__ void oem_chain(unsigned long long (&v)[M]) {
+template <int I, int J, int M> __device__ __forceinline__ void cmp_swap(unsigned (&v)[M]) {
+    const unsigned a = v[I], b = v[J];
+    v[I] = min(a, b);
+    v[J] = max(a, b);
+}
+template <int LO, int N, int R, int I, class T, int M> __device__ __forceinline__ void oem_chain(T (&v)[M]) {
     if constexpr (I + R < LO + N) {
         cmp_swap<I, I + R, M>(v);
-        oem_chain<LO, N, R, I + 2 * R, M>(v);
+        oem_chain<LO, N, R, I + 2 * R, T, M>(v);
     }
 }
 // merges the two sorted halves of the subsequence LO, LO+R, LO+2R, ... of v[LO .. LO+N)
-template <int LO, int N, int R, int M> __device__ __forceinline__ void oem_merge(unsigned long long (&v)[M]) {
+template <int LO, int N, int R, class T, int M> __device__ __forceinline__ void oem_merge(T (&v)[M]) {
     if constexpr (2 * R < N) {
-        oem_merge<LO, N, 2 * R, M>(v);
-        oem_merge<LO + R, N, 2 * R, M>(v);
-        oem_chain<LO, N, R, LO + R, M>(v);
+        oem_merge<LO, N, 2 * R, T, M>(v);
+        oem_merge<LO + R, N, 2 * R, T, M>(v);
+        oem_chain<LO, N, R, LO + R, T, M>(v);
     } else {
         cmp_swap<LO, LO + R, M>(v);
     }
 }
-template <int LO, int N, int M> __device__ __forceinline__ void oem_sort(unsigned long long (&v)[M]) {
+template <int LO, int N, class T, int M> __device__ __forceinline__ void oem_sort(T (&v)[M]) {
     if constexpr (N > 1) {
-        oem_sort<LO, N / 2, M>(v);
-        oem_sort<LO + N / 2, N / 2, M>(v);
-        oem_merge<LO, N, 1, M>(v);
+        oem_sort<LO, N / 2, T, M>(v);
+        oem_sort<LO + N / 2, N / 2, T, M>(v);
+        oem_merge<LO, N, 1, T, M>(v);
     }
 }
-template <int M> __device__ __forceinline__ void sort_regs(unsigned long long (&v)[M]) { oem_sort<0, M, M>(v); }
+template <class T, int M> __device__ __forceinline__ void sort_regs(T (&v)[M]) { oem_sort<0, M, T, M>(v); }
 
 // Sorts one line (stride `st` floats in shared memory) and returns the prefix sets of the
 // sorted order: pre[p] = positions of the p+1 best entries, packed two per word (16 bits
 // each) for M <= 16.
 template <int M> struct PreWords { static constexpr int value = (M == 32) ? 32 : M / 2; };
-template <int M>
-__device__ __forceinline__ void sort_line(const float* line, int st, unsigned (&pre)[PreWords<M>::value]) {
-    unsigned long long v[M];
-#pragma unroll
-    for (int k = 0; k < M; ++k) v[k] = sort_word(line[k * st], k);
-    sort_regs<M>(v);
+template <int M, class T>
+__device__ __forceinline__ void prefix_sets(const T (&v)[M], unsigned (&pre)[PreWords<M>::value]) {
     unsigned acc = 0u;
 #pragma unroll
     for (int p = 0; p < M; ++p) {
@@ -596,6 +617,28 @@ __device__ __forceinline__ void sort_line(const float* line, int st, unsigned (&
         if (M == 32) pre[p] = acc;
         else if (p % 2 == 0) pre[p / 2] = acc;
         else pre[p / 2] |= acc << 16;
+    }
+}
+template <int M>
+__device__ __forceinline__ void sort_line(const float* line, int st, unsigned (&pre)[PreWords<M>::value]) {
+    bool same_bucket;
+    {   // fast path: packed 32-bit words
+        unsigned w[M];
+#pragma unroll
+        for (int k = 0; k < M; ++k) w[k] = sort_word_packed(line[k * st], k);
+        sort_regs(w);
+        unsigned closest = 0xffffffffu;     // smallest difference pattern of two neighbours
+#pragma unroll
+        for (int p = 0; p + 1 < M; ++p) closest = min(closest, w[p] ^ w[p + 1]);
+        same_bucket = closest < 32u;
+        prefix_sets<M>(w, pre);
+    }
+    if (__any_sync(FULL, same_bucket)) {   // rare: two non-zero keys of a line within 2^-18 of each other
+        unsigned long long v[M];
+#pragma unroll
+        for (int k = 0; k < M; ++k) v[k] = sort_word(line[k * st], k);
+        sort_regs(v);
+        prefix_sets<M>(v, pre);
     }
 }
 
