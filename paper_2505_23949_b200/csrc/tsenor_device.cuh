@@ -531,9 +531,6 @@ __device__ __forceinline__ int load_key_panel(const float* __restrict__ src, int
 // both sorts have consumed the keys: key row i (M floats = 4M bytes) becomes
 //   M = 32 :  [0,4M) row prefixes of row i          (column prefixes: SmemLayout::cpre)
 //   M <= 16:  [0,2M) row prefixes of row i, [2M,4M) column prefixes of column i
-template <int M> struct RoundScratch {
-    unsigned int sel[M];          // current mask, one word per row (local search)
-};
 constexpr int CPRE_STRIDE = 33;   // words per column-prefix table at M = 32 (odd: conflict-free)
 
 // Strict order "key descending, index ascending" as one ascending u64.
@@ -682,11 +679,11 @@ template <int M> __device__ __forceinline__ unsigned transpose_bits(unsigned x, 
 //   ks, ws: shared-memory pointers to element (0,0) of the block's keys and
 //   |scores| (row stride WS); the key cells are overwritten.  cpre: this
 //   lane's column-prefix table when it does not fit in the key cells (M = 32).
-//   tb: the group's scratch; active: group has a block.
+//   active: group has a block.
 // Returns this lane's row of the mask (M bits).  flags accumulates DEV_* bits.
 template <class G>
-__device__ __forceinline__ unsigned round_block(float* ks, const float* ws, unsigned* cpre, RoundScratch<G::M>& tb,
-                                                int lane, bool active, int N, int ls_steps, int& flags) {
+__device__ __forceinline__ unsigned round_block(float* ks, const float* ws, unsigned* cpre, int lane, bool active,
+                                                int N, int ls_steps, int& flags) {
     constexpr int M = G::M;
     constexpr int WS = G::WS;
     constexpr unsigned GM = (M == 32) ? 0xffffffffu : ((1u << (M & 31)) - 1u);
@@ -726,7 +723,7 @@ __device__ __forceinline__ unsigned round_block(float* ks, const float* ws, unsi
     // available columns of my row; availC: available rows of my column.
     unsigned availR = active ? GM : 0u, availC = availR;
     int capR = active ? N : 0, capC = capR;
-    unsigned sel = 0u;
+    unsigned sel = 0u, selC = 0u;
     for (int round = 0; round < M * M; ++round) {
         if (!__any_sync(FULL, availR != 0u)) break;
         if (round == M * M - 1) flags |= DEV_INTERNAL;
@@ -736,6 +733,7 @@ __device__ __forceinline__ unsigned round_block(float* ks, const float* ws, unsi
         const unsigned takenR = pickR & transpose_bits<M>(pickC, i);   // columns taken in my row
         const unsigned takenC = transpose_bits<M>(takenR, i);          // rows taken in my column
         sel |= takenR;
+        selC |= takenC;
         capR -= __popc(takenR);
         capC -= __popc(takenC);
         // lines that just filled up drop out, and so do their entries
@@ -745,9 +743,9 @@ __device__ __forceinline__ unsigned round_block(float* ks, const float* ws, unsi
         availC = (capC == 0) ? 0u : (availC & ~takenC & ~fullR);
     }
 
-    // ---- local search (lines 7-13, Eq. 6).  Lane j' scans i' = 0..M-1.
-    tb.sel[i] = sel;
-    __syncwarp();
+    // ---- local search (lines 7-13, Eq. 6).  sel: my row of the mask (bits over columns);
+    // selC: my column (bits over rows).  Lane j' scans the rows i' that can form a valid
+    // triple with it: S[i'][j'] = 1 and S[i'][j] = 0, provided S[i][j'] = 0.
     bool stopped = !active;
     int steps = 0;
     for (int it = 0; it <= M * N; ++it) {
@@ -759,17 +757,16 @@ __device__ __forceinline__ unsigned round_block(float* ks, const float* ws, unsi
         const int di = work ? __ffs(rdef) - 1 : 0;   // lowest unsaturated row
         const int dj = work ? __ffs(cdef) - 1 : 0;   // lowest unsaturated column
         const int jp = i;                            // my candidate column j'
+        const unsigned col_dj = __shfl_sync(FULL, selC, dj, M);          // rows that hold column j
+        unsigned cand = (work && !((selC >> di) & 1u)) ? (selC & ~col_dj) : 0u;
         float best = __int_as_float(0xff800000);
         int bi = 0x7fffffff;
-        if (work && !((tb.sel[di] >> jp) & 1u)) {
-            const float w_ijp = ws[di * WS + jp];
-#pragma unroll 4
-            for (int ip = 0; ip < M; ++ip) {
-                const unsigned s = tb.sel[ip];
-                const bool valid = ((s >> jp) & 1u) && !((s >> dj) & 1u);
-                const float sc = __fsub_rn(__fadd_rn(w_ijp, ws[ip * WS + dj]), ws[ip * WS + jp]);
-                if (valid && sc > best) { best = sc; bi = ip; }
-            }
+        const float w_ijp = ws[di * WS + jp];
+        while (cand) {                               // ascending i': ties keep the smallest
+            const int ip = __ffs(cand) - 1;
+            cand &= cand - 1u;
+            const float sc = __fsub_rn(__fadd_rn(w_ijp, ws[ip * WS + dj]), ws[ip * WS + jp]);
+            if (sc > best) { best = sc; bi = ip; }
         }
         int bflat = (bi == 0x7fffffff) ? 0x7fffffff : bi * M + jp;
 #pragma unroll
@@ -787,13 +784,11 @@ __device__ __forceinline__ unsigned round_block(float* ks, const float* ws, unsi
                 const int ip = bflat / M, jq = bflat % M;
                 if (i == ip) sel = (sel & ~(1u << jq)) | (1u << dj);
                 if (i == di) { sel |= 1u << jq; --capR; }
-                if (i == dj) --capC;
+                if (i == jq) selC = (selC & ~(1u << ip)) | (1u << di);
+                if (i == dj) { selC |= 1u << ip; --capC; }
                 ++steps;
             }
         }
-        __syncwarp();
-        tb.sel[i] = sel;
-        __syncwarp();
     }
     if (active && (capR != 0 || capC != 0)) flags |= DEV_UNDERFILLED;
     return sel;
@@ -825,7 +820,6 @@ template <class G, int MODE> struct SmemLayout {
     static constexpr int M = G::M;
     float w[M * G::WS];
     float k[M * G::WS];
-    RoundScratch<M> tb[WARPS * G::GPW];
     unsigned int bits[M * G::WORDS];
     unsigned int cpre[(M == 32) ? WARPS * 32 * CPRE_STRIDE : 1];   // column-prefix tables (M = 32)
 };
@@ -833,7 +827,6 @@ template <class G> struct SmemLayout<G, 1> {   // Algorithm 1 alone: score panel
     static constexpr int M = G::M;
     float w[M * G::WS];
     float k[WARPS * 32 * G::T::MR * G::T::MC];
-    RoundScratch<M> tb[1];
     unsigned int bits[1];
     unsigned int cpre[1];
 };
@@ -961,13 +954,12 @@ __global__ void __launch_bounds__(WARPS * 32, MinBlocks<M, V>::value) tsenor_ker
     // ---- Algorithm 2 and the mask writer
     if (MODE != 1) {
         const int grp = lane / M;
-        RoundScratch<M>& tb = sm.tb[warp * G::GPW + grp];
 #pragma unroll 1
         for (int pass = 0; pass < G::PASSES; ++pass) {
             const int blk = warp * G::BPW + pass * G::GPW + grp;
             const bool active = (pass * G::GPW + grp < G::BPW) && blk * M < valid_cols;
             const unsigned row_bits =
-                round_block<G>(sm.k + blk * M, sm.w + blk * M, sm.cpre + (warp * 32 + lane) * CPRE_STRIDE, tb, lane,
+                round_block<G>(sm.k + blk * M, sm.w + blk * M, sm.cpre + (warp * 32 + lane) * CPRE_STRIDE, lane,
                                active, P.N, P.ls_steps, flags);
             if (active) {
                 const int off = blk * M;
