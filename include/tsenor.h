@@ -52,8 +52,11 @@ enum {
 
 /* Bits OR-ed into *dev_status by the kernels. */
 enum {
-    TSENOR_DEV_NONFINITE_SCORE = 1, /* a score or key was NaN/inf; masks of the
-                                       blocks holding one are unspecified      */
+    TSENOR_DEV_NONFINITE_SCORE = 1, /* a score was NaN/inf (masks of the blocks
+                                       holding one are unspecified), or a key
+                                       given to tsenor_round was NaN (it orders
+                                       last; infinite keys are legal and not
+                                       flagged)                                */
     TSENOR_DEV_UNDERFILLED = 2,     /* some block ended with fewer than N per
                                        line (only possible with ls_steps >= 0
                                        or non-finite input)                    */

@@ -18,6 +18,19 @@ constexpr int WARPS = 4;  // warps per CTA
 
 enum : int { DEV_NONFINITE = 1, DEV_UNDERFILLED = 2, DEV_INTERNAL = 4 };
 
+// Checked build flavour (-DTSENOR_BOUNDS, a second library built from the same sources): every
+// data-dependent or computed index of the loaders, the rounding tables, the local search and the
+// writers is tested against the extent of its array before the access; a bad one ORs
+// DEV_INTERNAL into the status word and the access is skipped (nothing traps, nothing faults).
+// It stands in for a memory checker on machines where none can be run.  In the normal build
+// TS_CHECK(x) is the constant true and costs nothing.
+#ifdef TSENOR_BOUNDS
+__shared__ int g_bounds_flags;
+#define TS_CHECK(cond) ((cond) ? true : (atomicOr(&tsenor::g_bounds_flags, tsenor::DEV_INTERNAL), false))
+#else
+#define TS_CHECK(cond) true
+#endif
+
 // ---------------------------------------------------------------------------
 // Dykstra register layout.  A block is spread over LPB = PR*PC lanes arranged
 // as PR x PC; each lane keeps an MR x MC sub-tile.  Row sums are reduced over
@@ -54,6 +67,7 @@ template <int M_, int V_> struct Geom {
     static constexpr int WORDS = PANEL / 32;         // mask words per panel row
     static_assert(T::MR >= T::PC && T::MC >= T::PR && T::MC % 2 == 0 && (T::MR * T::MC) % 4 == 0, "tile shape");
     static_assert(T::PR * T::MR == M && T::PC * T::MC == M, "tile covers the block");
+    static_assert(WARPS * 32 * T::MR * T::MC <= M * WS, "the per-warp stashes of t0 fit in the key panel");
 };
 
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -454,6 +468,9 @@ __device__ __forceinline__ float4 load_score_quad(const ScoreSrc& S, int64_t r, 
                        score_of(S.kind, w.z, v.z, S.scalar, cv.z), score_of(S.kind, w.w, v.w, S.scalar, cv.w));
 }
 
+__device__ __forceinline__ int any_nan(const float4& v) {
+    return !(v.x == v.x) | !(v.y == v.y) | !(v.z == v.z) | !(v.w == v.w);
+}
 __device__ __forceinline__ int any_nonfinite(const float4& v) {
     return !(fabsf(v.x) <= 3.4028234e38f) | !(fabsf(v.y) <= 3.4028234e38f) |
            !(fabsf(v.z) <= 3.4028234e38f) | !(fabsf(v.w) <= 3.4028234e38f);
@@ -472,14 +489,18 @@ template <int M> struct PanelMap {
     int64_t r0, c0;        // wide: origin of the panel
     int64_t first;         // tall: first block (= block row) of the panel
     int valid_cols;        // columns of the shared-memory panel that hold blocks
+    int64_t rows, cols;    // extent of the matrix
+    __device__ __forceinline__ bool holds_quad(int64_t r, int64_t c) const {
+        return r >= 0 && r < rows && c >= 0 && c + 4 <= cols;
+    }
     __device__ __forceinline__ int64_t row(int r, int c) const { return tall ? (first + c / M) * M + r : r0 + r; }
     __device__ __forceinline__ int64_t col(int c) const { return tall ? (int64_t)(c % M) : c0 + c; }
 };
 
 // ---------------------------------------------------------------------------
 // Panel loaders: an M x PANEL panel into shared memory, coalesced, vector
-// loads when the addresses allow it.  Return non-zero if a non-finite value
-// was seen by this thread.
+// loads when the addresses allow it.  Return non-zero if this thread saw a
+// non-finite score, respectively a NaN key.
 // ---------------------------------------------------------------------------
 template <class G>
 __device__ __forceinline__ int load_score_panel(const ScoreSrc& S, const PanelMap<G::M>& pm,
@@ -490,10 +511,13 @@ __device__ __forceinline__ int load_score_panel(const ScoreSrc& S, const PanelMa
     for (int idx = threadIdx.x; idx < M * V; idx += WARPS * 32) {
         const int r = idx / V, c = (idx % V) * 4;
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (c < pm.valid_cols) v = load_score_quad(S, pm.row(r, c), pm.col(c));  // a quad is all in or all out
+        if (c < pm.valid_cols && TS_CHECK(pm.holds_quad(pm.row(r, c), pm.col(c))))
+            v = load_score_quad(S, pm.row(r, c), pm.col(c));  // a quad is all in or all out
         bad |= any_nonfinite(v);
-        float* d = dst + r * G::WS + c;
-        d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
+        if (TS_CHECK(r < M && c + 4 <= G::PANEL)) {
+            float* d = dst + r * G::WS + c;
+            d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
+        }
     }
     return bad;
 }
@@ -507,14 +531,16 @@ __device__ __forceinline__ int load_key_panel(const float* __restrict__ src, int
     for (int idx = threadIdx.x; idx < M * V; idx += WARPS * 32) {
         const int r = idx / V, c = (idx % V) * 4;
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (c < pm.valid_cols) {
+        if (c < pm.valid_cols && TS_CHECK(pm.holds_quad(pm.row(r, c), pm.col(c)))) {
             const float* p = src + pm.row(r, c) * ld + pm.col(c);
             if (vec_ok) v = __ldg(reinterpret_cast<const float4*>(p));
             else v = make_float4(__ldg(p), __ldg(p + 1), __ldg(p + 2), __ldg(p + 3));
         }
-        bad |= any_nonfinite(v);
-        float* d = dst + r * G::WS + c;
-        d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
+        bad |= any_nan(v);          // infinite keys have a place in the order; NaN keys are flagged
+        if (TS_CHECK(r < M && c + 4 <= G::PANEL)) {
+            float* d = dst + r * G::WS + c;
+            d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
+        }
     }
     return bad;
 }
@@ -641,6 +667,7 @@ __device__ __forceinline__ void sort_line(const float* line, int st, unsigned (&
 
 // Prefix p of a stored table (tab points to the table's first byte).
 template <int M> __device__ __forceinline__ unsigned prefix_at(const void* tab, int p) {
+    if (!TS_CHECK(p >= 0 && p < M)) return 0u;
     if (M == 32) return static_cast<const unsigned*>(tab)[p];
     return static_cast<const unsigned short*>(tab)[p];
 }
@@ -757,14 +784,16 @@ __device__ __forceinline__ unsigned round_block(float* ks, const float* ws, unsi
         const int di = work ? __ffs(rdef) - 1 : 0;   // lowest unsaturated row
         const int dj = work ? __ffs(cdef) - 1 : 0;   // lowest unsaturated column
         const int jp = i;                            // my candidate column j'
-        const unsigned col_dj = __shfl_sync(FULL, selC, dj, M);          // rows that hold column j
-        unsigned cand = (work && !((selC >> di) & 1u)) ? (selC & ~col_dj) : 0u;
+        const bool lines_ok = TS_CHECK(di >= 0 && di < M && dj >= 0 && dj < M);
+        const unsigned col_dj = __shfl_sync(FULL, selC, lines_ok ? dj : 0, M);   // rows that hold column j
+        unsigned cand = (work && lines_ok && !((selC >> di) & 1u)) ? (selC & ~col_dj & GM) : 0u;
         float best = __int_as_float(0xff800000);
         int bi = 0x7fffffff;
-        const float w_ijp = ws[di * WS + jp];
+        const float w_ijp = lines_ok ? ws[di * WS + jp] : 0.0f;
         while (cand) {                               // ascending i': ties keep the smallest
             const int ip = __ffs(cand) - 1;
             cand &= cand - 1u;
+            if (!TS_CHECK(ip < M)) continue;
             const float sc = __fsub_rn(__fadd_rn(w_ijp, ws[ip * WS + dj]), ws[ip * WS + jp]);
             if (sc > best) { best = sc; bi = ip; }
         }
@@ -780,6 +809,8 @@ __device__ __forceinline__ unsigned round_block(float* ks, const float* ws, unsi
                 stopped = true;
             } else if (ls_steps >= 0 && !(best > 0.0f)) {
                 stopped = true;                   // paper-strict loop: improving swaps only
+            } else if (!TS_CHECK(bflat >= 0 && bflat < M * M)) {
+                stopped = true;
             } else {
                 const int ip = bflat / M, jq = bflat % M;
                 if (i == ip) sel = (sel & ~(1u << jq)) | (1u << dj);
@@ -845,6 +876,11 @@ __global__ void __launch_bounds__(WARPS * 32, MinBlocks<M, V>::value) tsenor_ker
     const int64_t panel = blockIdx.x;
     PanelMap<M> pm;
     pm.tall = P.tall;
+    pm.rows = P.rows; pm.cols = P.cols;
+#ifdef TSENOR_BOUNDS
+    if (threadIdx.x == 0) g_bounds_flags = 0;
+    __syncthreads();
+#endif
     if (P.tall) {
         constexpr int NB = G::PANEL / M;
         const int64_t left = P.rows / M - panel * NB;
@@ -883,7 +919,7 @@ __global__ void __launch_bounds__(WARPS * 32, MinBlocks<M, V>::value) tsenor_ker
 #pragma unroll
             for (int b = 0; b < MC; ++b) {
                 const int col = blk * M + lc * MC + (b ^ gc);
-                t[a][b] = sm.w[row * G::WS + col];
+                t[a][b] = TS_CHECK(row < M && col < G::PANEL) ? sm.w[row * G::WS + col] : 0.0f;
                 m = fmaxf(m, t[a][b]);
             }
             mx[a] = m;
@@ -937,7 +973,9 @@ __global__ void __launch_bounds__(WARPS * 32, MinBlocks<M, V>::value) tsenor_ker
                     for (int b = 0; b < MC; ++b) {
                         const int pc = blk * M + lc * MC + (b ^ gc);
                         const int64_t row = pm.row(lr * MR + (a ^ gr), pc), col = pm.col(pc);
-                        P.plan[row * P.ld_plan + col] = P.plan_is_log ? t[a][b] * 0.6931471805599453f : exp2f(t[a][b]);
+                        if (TS_CHECK(row >= 0 && row < P.rows && col >= 0 && col < P.cols))
+                            P.plan[row * P.ld_plan + col] =
+                                P.plan_is_log ? t[a][b] * 0.6931471805599453f : exp2f(t[a][b]);
                     }
             }
         } else {
@@ -946,7 +984,8 @@ __global__ void __launch_bounds__(WARPS * 32, MinBlocks<M, V>::value) tsenor_ker
             for (int a = 0; a < MR; ++a)
 #pragma unroll
                 for (int b = 0; b < MC; ++b)
-                    sm.k[(lr * MR + (a ^ gr)) * G::WS + blk * M + lc * MC + (b ^ gc)] = t[a][b];
+                    if (TS_CHECK(lr * MR + (a ^ gr) < M && blk * M + lc * MC + (b ^ gc) < G::PANEL))
+                        sm.k[(lr * MR + (a ^ gr)) * G::WS + blk * M + lc * MC + (b ^ gc)] = t[a][b];
         }
         __syncwarp();
     }
@@ -958,10 +997,11 @@ __global__ void __launch_bounds__(WARPS * 32, MinBlocks<M, V>::value) tsenor_ker
         for (int pass = 0; pass < G::PASSES; ++pass) {
             const int blk = warp * G::BPW + pass * G::GPW + grp;
             const bool active = (pass * G::GPW + grp < G::BPW) && blk * M < valid_cols;
+            if (!TS_CHECK(blk * M + M <= G::PANEL)) continue;     // warp-uniform up to the group
             const unsigned row_bits =
                 round_block<G>(sm.k + blk * M, sm.w + blk * M, sm.cpre + (warp * 32 + lane) * CPRE_STRIDE, lane,
                                active, P.N, P.ls_steps, flags);
-            if (active) {
+            if (active && TS_CHECK(blk * M / 32 < G::WORDS)) {
                 const int off = blk * M;
                 if (M == 32) sm.bits[(lane % M) * G::WORDS + off / 32] = row_bits;
                 else atomicOr(&sm.bits[(lane % M) * G::WORDS + off / 32], row_bits << (off % 32));
@@ -973,16 +1013,23 @@ __global__ void __launch_bounds__(WARPS * 32, MinBlocks<M, V>::value) tsenor_ker
             constexpr unsigned GM = (M == 32) ? 0xffffffffu : ((1u << (M & 31)) - 1u);
             for (int idx = threadIdx.x; idx < valid_cols; idx += WARPS * 32) {
                 const int blk = idx / M, r = idx % M;
-                P.bits[((pm.first + blk) * M + r) * P.wpr] = (sm.bits[r * G::WORDS + (blk * M) / 32] >> ((blk * M) % 32)) & GM;
+                if (TS_CHECK((pm.first + blk) * M + r < P.rows && (blk * M) / 32 < G::WORDS))
+                    P.bits[((pm.first + blk) * M + r) * P.wpr] =
+                        (sm.bits[r * G::WORDS + (blk * M) / 32] >> ((blk * M) % 32)) & GM;
             }
         } else {
             const int nwords = (valid_cols + 31) / 32;
             for (int idx = threadIdx.x; idx < M * G::WORDS; idx += WARPS * 32) {
                 const int r = idx / G::WORDS, wd = idx % G::WORDS;
-                if (wd < nwords) P.bits[(pm.r0 + r) * P.wpr + pm.c0 / 32 + wd] = sm.bits[idx];
+                if (wd < nwords && TS_CHECK(pm.r0 + r < P.rows && pm.c0 / 32 + wd < P.wpr))
+                    P.bits[(pm.r0 + r) * P.wpr + pm.c0 / 32 + wd] = sm.bits[idx];
             }
         }
     }
+#ifdef TSENOR_BOUNDS
+    __syncthreads();
+    flags |= g_bounds_flags;
+#endif
     flags = __reduce_or_sync(FULL, flags);
     if (flags && lane == 0 && P.status) atomicOr(P.status, flags);
 }

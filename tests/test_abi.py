@@ -31,6 +31,13 @@ def test_library_exports_every_declared_symbol(lib):
         assert getattr(lib, name) is not None
 
 
+def test_checked_flavour_builds_and_exports_the_same_symbols():
+    import ctypes
+    checked = ctypes.CDLL(ts_build.build(bounds=True))
+    for name in _declared_functions():
+        assert getattr(checked, name) is not None
+
+
 def test_host_arithmetic_and_messages(lib):
     assert [lib.tsenor_mask_words_per_row(c) for c in (0, 1, 32, 33, 4096)] == [0, 1, 1, 2, 128]
     for code in (0, -1, -2, -3, -4, -5):
