@@ -36,8 +36,8 @@ NOMINAL_SM_MHZ = 1965.0
 # summarised in PROFILE_SUMMARY (not measured by this script: they go stale if the kernel changes
 # and the capture is not repeated, which is why the JSON line names their source).
 PROFILE_SUMMARY = "profiles/tsenor_kernel_m32_solve_config4_up.md"
-NCU_DRAM_BYTES_PER_LAUNCH = 244.09e6      # dram__bytes_read.sum + dram__bytes_write.sum
-NCU_WARP_INST_PER_BLOCK_ITER = 170.0      # smsp__inst_executed.sum / (57,344 blocks x 300 iterations)
+NCU_DRAM_BYTES_PER_LAUNCH = 244.98e6      # dram__bytes_read.sum + dram__bytes_write.sum
+NCU_WARP_INST_PER_BLOCK_ITER = 145.6      # smsp__inst_executed.sum / (57,344 blocks x 300 iterations)
 
 
 def fp32_lane_ops_per_block(M, T):
