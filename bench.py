@@ -145,7 +145,7 @@ def aggregate_rate(units_per_rank_per_step, steps, world, elapsed_ms):
 
 
 WORKLOADS = ("config4", "config0", "config1", "config2", "config3", "config5", "admm", "admm_small", "wanda",
-             "sparsegpt", "config4_earlyexit")
+             "sparsegpt", "config4_earlyexit", "config4_bf16")
 EARLY_EXIT_EPS = 1e-3
 
 
@@ -158,6 +158,8 @@ class Job:
         self.rows, self.cols = arrays["w"].shape
         self.blocks = (self.rows // M) * (self.cols // M)
         self.score_bytes = self.rows * self.cols * 4          # fp32 scores the mask is computed from
+        if kind == "abs_bf16":
+            self.score_bytes = self.rows * self.cols * 2
         self.h2d_bytes = sum(a.nbytes for a in arrays.values())
 
 
@@ -170,6 +172,13 @@ def make_jobs(workload, index):
     if workload == "config4_earlyexit":   # the headline matrices in the stopping-test mode (non-parity)
         return [Job(w.name, w.N, w.M, {"w": w.scores}, kind="abs_ee", ee_eps=EARLY_EXIT_EPS)
                 for w in (synth.config(4, index=index, part="up"), synth.config(4, index=index, part="down"))]
+    if workload == "config4_bf16":        # the headline matrices handed over as bf16 (half the bytes to move)
+        import torch
+        jobs = []
+        for w in (synth.config(4, index=index, part="up"), synth.config(4, index=index, part="down")):
+            wb = torch.from_numpy(w.scores).to(torch.bfloat16)
+            jobs.append(Job(w.name + "-bf16", w.N, w.M, {"w": wb.view(torch.int16).numpy()}, kind="abs_bf16"))
+        return jobs
     if workload == "config1":     # 16 different matrices per step: a single 50 us launch between two
         jobs = []                 # event records would time the host's launch path, not the kernel
         for k in range(16):
@@ -232,6 +241,8 @@ WORKLOAD_TEXT = {
     "config4_earlyexit": "config 4 matrices in the stopping-test mode of Algorithm 1 (NOT the parity contract): a "
                          "block stops once its marginal violation is below 1e-3 (tested every 4 iterations, at most "
                          "300); roofline figures count the iterations actually run",
+    "config4_bf16": "config 4 with the weights handed over in bf16 (rounded from the fp32 draw, widened exactly "
+                    "to fp32 in the block loader): same shapes, 16:32, half the bytes per matrix",
     "wanda": "Wanda scores |W_ij| a_j computed in the loader from bf16 W (4096x4096) and fp32 a_j, 8:16",
     "sparsegpt": "SparseGPT column groups: eight 14336x32 slabs solved one after the other (latency case: 448 "
                  "blocks per call), scores |W_ij / d_j| computed in the loader, 16:32",
@@ -269,6 +280,9 @@ def oracle_sample(job, blocks_wanted):
         full = oracle.scores(oracle.SCORES_COLMUL, wf, colvec=job.arrays["a"])
     elif job.kind == "coldiv":
         full = oracle.scores(oracle.SCORES_COLDIV, w, colvec=job.arrays["d"])
+    elif job.kind == "abs_bf16":
+        import torch
+        full = torch.from_numpy(w).view(torch.bfloat16).to(torch.float32).numpy()
     else:
         full = w
     return np.ascontiguousarray(full[: nrows * M]), nrows * per_row, float(full.max())
@@ -385,6 +399,8 @@ def run_cuda(args, rank, world, local_rank):
                 return ts.Scores(ts.SCORES_COLMUL, t["w"].view(torch.bfloat16), colvec=t["a"])
             if j.kind == "coldiv":
                 return ts.Scores(ts.SCORES_COLDIV, t["w"], colvec=t["d"])
+            if j.kind == "abs_bf16":
+                return ts.Scores(ts.SCORES_ABS, t["w"].view(torch.bfloat16))
             if j.kind == "abs_ee":
                 return ts.Scores(ts.SCORES_ABS, t["w"], early_exit_eps=j.ee_eps, iters_out=self.iters_run)
             return ts.Scores(ts.SCORES_ABS, t["w"])
