@@ -330,8 +330,8 @@ def run_reference(args, rank):
     cfg, _ = workload_config(args.workload, jobs)
     # calibrate on one block row, then size each step so the whole run stays within minutes
     rate, _, _, cores = time_oracle(job, 128)
-    budget_s = 150.0
-    per_step = int(max(128, min(8192, rate * budget_s / max(1, args.steps + args.warmup))))
+    limit_s = 150.0
+    per_step = int(max(128, min(8192, rate * limit_s / max(1, args.steps + args.warmup))))
     sample, nblk, mx = oracle_sample(job, per_step)
     tau = synth.default_tau(mx)
     for _ in range(args.warmup):
