@@ -12,7 +12,9 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libtsenor.so")
+# The library beside this file; TSENOR_LIBRARY selects another build of the same ABI (for instance
+# the checked flavour libtsenor_bounds.so, to run a whole test suite with every index tested).
+LIB_PATH = os.environ.get("TSENOR_LIBRARY") or os.path.join(_HERE, "libtsenor.so")
 
 OK, ERR_NULL, ERR_SHAPE, ERR_NM, ERR_ARG, ERR_CUDA = 0, -1, -2, -3, -4, -5
 DEV_NONFINITE_SCORE, DEV_UNDERFILLED, DEV_INTERNAL = 1, 2, 4
