@@ -86,3 +86,18 @@ def test_output_tensor_checks_raise_before_anything_reaches_the_library():
         with pytest.raises(TypeError):
             ts._out(bad, "mask_out", kw["dtype"], kw["device"])
     assert ts._out(None, "status", torch.int32, "cuda:0") is None
+
+
+def test_header_is_plain_c(tmp_path):
+    """include/tsenor.h compiles as C11 and as C++ on its own (no CUDA headers needed by a caller)."""
+    import subprocess
+    src = tmp_path / "use_header.c"
+    src.write_text('#include "tsenor.h"\n'
+                   '#include <string.h>\n'
+                   'int use(void) { tsenor_scores_t s; memset(&s, 0, sizeof s); s.kind = TSENOR_SCORES_ABS; '
+                   'return (int)tsenor_mask_words_per_row(64) + s.kind + TSENOR_LAYOUT_AUTO; }\n')
+    inc = os.path.join(ROOT, "include")
+    subprocess.run(["gcc", "-std=c11", "-Wall", "-Wextra", "-Werror", "-I", inc, "-c", str(src), "-o",
+                    str(tmp_path / "c.o")], check=True)
+    subprocess.run(["g++", "-std=c++17", "-Wall", "-Wextra", "-Werror", "-x", "c++", "-I", inc, "-c", str(src), "-o",
+                    str(tmp_path / "cc.o")], check=True)
